@@ -1,0 +1,200 @@
+/*
+ * entwine.h - C ABI of the B200 (sm_100a) fused GEMM-ReduceScatter of a tensor-parallel
+ * row-parallel linear layer, run on one GPU as a one-rank emulation of W logical ranks
+ * (Entwine: interleaved tile production + tile-level flags + SM-based communication).
+ *
+ * Conventions
+ *   - Every function returns an int: ENTWINE_OK (0) or a negative ENTWINE_ERR_* code.
+ *     Nothing throws across this boundary; nothing traps or hangs the device: every
+ *     device-side wait is bounded and reports through the plan's status word.
+ *   - "device pointer" = global memory of the current CUDA device, 16-byte aligned,
+ *     valid until the stream has finished the call.  "host pointer" = ordinary host
+ *     memory.  The library never takes ownership of caller buffers.
+ *   - No function synchronises the device unless its comment says so.
+ *   - A plan is not thread-safe; calls on one plan must be issued from one thread and are
+ *     serialised on the device by stream order (use one stream per plan).
+ *
+ * Notation (paper Sec. 3.1 / 4.2): R = M/W rows per output partition; reduction tile
+ * 128x128; producer block 128 x BN with BN in {128,256}; cpb = BN/128; nTn = N/128;
+ * Q = (R/128)*nTn tiles per partition; P_blk = (M/128)*(N/BN) producer blocks; r = the
+ * emulated rank; x = number of consumer (communication) task lists.
+ *
+ * Data layout (all bf16, row-major, contiguous)
+ *   A             [M, K_local]
+ *   B             [N, K_local]   the rank's shard of the layer weight (K contiguous), so the
+ *                                rank's partial output is C = A . B^T, [M, N]
+ *   peer_partials [W-1, M, N]    incoming partial outputs of the other ranks in ascending
+ *                                rank order (slot q(w) = w < r ? w : w-1).  Only rows
+ *                                [r*R, (r+1)*R) of each are read (Sec. 4.1: contributions
+ *                                sit at matching offsets in every rank's buffer).
+ *   out_shard     [R, N]         the reduced output partition of rank r
+ *   send_bufs     [W-1, R, N]    slot q(d) receives rows [d*R,(d+1)*R) of C: what rank r
+ *                                contributes to destination d (stands in for peer memory)
+ */
+#ifndef ENTWINE_H_
+#define ENTWINE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct entwine_plan_s* entwine_plan_t;
+
+/* Producer tile orders (Sec. 3.1 and Fig. 1). */
+enum {
+  ENTWINE_ORDER_ROW_MAJOR   = 0, /* partition-grouped: all blocks of partition 0, then 1, ... */
+  ENTWINE_ORDER_INTERLEAVED = 1  /* Eq. 1: d = p mod W, l = floor(p / W)                      */
+};
+
+enum {
+  ENTWINE_OK            =  0,
+  ENTWINE_ERR_INVALID   = -1, /* bad shape, argument, option or call order                  */
+  ENTWINE_ERR_RESOURCES = -2, /* not enough SMs / shared memory for a co-resident launch     */
+  ENTWINE_ERR_CUDA      = -3, /* a CUDA call failed, or there is no CUDA device              */
+  ENTWINE_ERR_TIMEOUT   = -4, /* a device-side wait ran out of its budget                    */
+  ENTWINE_ERR_INTERNAL  = -5  /* a device-side index check failed                            */
+};
+
+/* Option keys for entwine_set_option. Options marked [pre] must be set before the first
+ * launch of the plan; the others may change between launches. */
+enum {
+  ENTWINE_OPT_RANK            = 1, /* [pre] emulated rank r, 0 <= r < W (default 0)             */
+  ENTWINE_OPT_BLOCK_N         = 2, /* [pre] producer block width BN: 128 or 256 (default 256)   */
+  ENTWINE_OPT_WAIT_BUDGET_NS  = 3, /* budget of every device-side flag wait (default 2e9 ns)    */
+  ENTWINE_OPT_TAIL_HELP       = 4, /* 1 (default): producer CTAs that have finished their last
+                                      block take tasks from the consumer lists (the one-launch
+                                      analogue of the shared SM pool, Sec. 3.2 "Resource reuse");
+                                      0: strict static partition (Sec. 5.3.3's other arm)        */
+  ENTWINE_OPT_WITHHOLD_PEER   = 5, /* host-side fault injection: value = w*2^32 + t withholds the
+                                      pre-published flag of peer rank w for tile t; -1 restores
+                                      all peer flags (default)                                   */
+  ENTWINE_OPT_NUM_SMS         = 6, /* [pre] override the SM count used for planning (testing
+                                      without a device; default: the device's SM count, 148 if
+                                      there is no device)                                        */
+  ENTWINE_OPT_POISON_PARTIAL  = 7  /* 1: fill the partial-output workspace with NaN patterns
+                                      before each launch (ordering stress test; default 0)       */
+};
+
+/* What entwine_plan_export can write.  Integer tables, host memory, for bit-exact diffs. */
+enum {
+  ENTWINE_EXPORT_COUNTS      = 0, /* int64[16]: P_blk, Q, cpb, x, n_tasks, n_reduce, n_push,
+                                     flags_published, peer_flags_prepublished, min_flag_reads,
+                                     bytes_peer_read, bytes_own_read, bytes_push_write,
+                                     bytes_out_write, n_gemm_ctas, n_comm_ctas               */
+  ENTWINE_EXPORT_ORDER       = 1, /* int32[P_blk][4]: mb, nb, d, l per logical position p     */
+  ENTWINE_EXPORT_TILES       = 2, /* int32[P_blk][cpb]: tile indices covered by block p       */
+  ENTWINE_EXPORT_FLAG_SEQ    = 3, /* int32[P_blk*cpb][3]: (src=r, d, t) at k = p*cpb + c      */
+  ENTWINE_EXPORT_LIST_OFFS   = 4, /* int32[x+1]: rows of TASKS that belong to list j          */
+  ENTWINE_EXPORT_TASKS       = 5, /* int64[n_tasks][8]: kind(0 reduce,1 push), d, t, k, list,
+                                     src_off, dst_slot(-1 for reduce), dst_off  (elements)    */
+  ENTWINE_EXPORT_PEER_OFFS   = 6  /* int64[n_reduce][W-1]: element offsets into peer_partials */
+};
+
+/*
+ * entwine_plan - validate a problem and build its schedule (Sec. 3.1 Eq. 1, Sec. 3.2).
+ *   M, N, K_local  GEMM extents of the emulated rank (C[M,N] = A[M,K_local] . B[N,K_local]^T)
+ *   W              number of logical ranks, >= 2
+ *   tile_order     ENTWINE_ORDER_*
+ *   n_comm_sms     SMs dedicated to communication CTAs (the communication budget x,
+ *                  Sec. 3.2); 0 = non-overlapped use of all SMs: every CTA first produces,
+ *                  then consumes (Sec. 5.3.2's baseline)
+ * Requirements (Sec. 4.1): M % (128*W) == 0, N % 128 == 0 (and N % BN == 0 at launch),
+ * K_local % 16 == 0, 0 <= n_comm_sms < number of SMs.
+ * The plan owns the partial-output workspace C[M,N] (bf16), the flag arrays, the device
+ * copies of the task tables and a status block; they are allocated with cudaMalloc at the
+ * first launch (so do the first launch outside stream capture) and reused by every later
+ * launch (Sec. 4.1).  Without a CUDA device the plan is host-only: tables can be exported,
+ * launches return ENTWINE_ERR_CUDA.
+ * Writes the handle to *plan.  Errors: ENTWINE_ERR_INVALID.
+ */
+int entwine_plan(entwine_plan_t* plan, int64_t M, int64_t N, int64_t K_local, int W,
+                 int tile_order, int n_comm_sms);
+
+/* entwine_set_option - see ENTWINE_OPT_*.  Errors: ENTWINE_ERR_INVALID (unknown key, bad
+ * value, or a [pre] option after the first launch). */
+int entwine_set_option(entwine_plan_t plan, int key, int64_t value);
+
+/*
+ * entwine_gemm_rs - one fused GEMM-ReduceScatter call of the emulated rank, enqueued on
+ * `stream` (a cudaStream_t passed as void*; NULL = the default stream).  One kernel launch:
+ * producer CTAs run the tcgen05 GEMM over the plan's block order and publish one flag per
+ * finished 128x128 tile (Sec. 3.1, Sec. 4.2); consumer CTAs on the dedicated SMs poll the
+ * flags, copy non-owned tiles to send_bufs and reduce owned tiles with the W-1 incoming
+ * partials into out_shard (ReduceTile, Sec. 4.2: start from the local contribution, add the
+ * peers in ascending rank order in fp32, single writer).
+ * All five pointers are device pointers (layouts above).  Returns after enqueueing.
+ * Errors: ENTWINE_ERR_INVALID (null / misaligned pointer), ENTWINE_ERR_RESOURCES,
+ * ENTWINE_ERR_CUDA; a timeout or index failure of an earlier launch that
+ * entwine_last_status has not yet collected is returned as ENTWINE_ERR_TIMEOUT /
+ * ENTWINE_ERR_INTERNAL by that later query, never by a trap.
+ */
+int entwine_gemm_rs(entwine_plan_t plan, const void* A, const void* B,
+                    const void* peer_partials, void* out_shard, void* send_bufs,
+                    void* stream);
+
+/*
+ * entwine_gemm_rs_host - the same call for HOST buffers (same layouts): copies A, B and
+ * rows [r*R,(r+1)*R) of each peer partial to plan-owned device staging buffers, runs the
+ * fused kernel, copies out_shard and send_bufs back and synchronises the plan's internal
+ * stream before returning.  Pinned host memory makes the copies asynchronous with each
+ * other but is not required.  Errors as entwine_gemm_rs, plus a pending device status.
+ */
+int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B,
+                         const void* peer_partials, void* out_shard, void* send_bufs);
+
+/*
+ * entwine_gemm_only - the producer alone on all SMs (no consumer work): fills the plan's
+ * partial-output workspace and publishes the flags.  Gives the uncontended GEMM time of the
+ * overlap-efficiency ratio (Sec. 5.2.1, App. C).  A, B device pointers.
+ */
+int entwine_gemm_only(entwine_plan_t plan, const void* A, const void* B, void* stream);
+
+/*
+ * entwine_comm_only - the consumer alone with every input already available (App. A):
+ * all flags are treated as published and n_ctas communication CTAs (0 = one per SM) walk
+ * the task lists.  partial = device pointer to a bf16 C[M,N] to consume, or NULL for the
+ * plan's own workspace (as left by the last producer run).  With partial produced by a
+ * library GEMM this is the second half of the unfused GEMM-then-ReduceScatter sequence.
+ */
+int entwine_comm_only(entwine_plan_t plan, const void* partial, const void* peer_partials,
+                      void* out_shard, void* send_bufs, int n_ctas, void* stream);
+
+/*
+ * entwine_read_partial - copy the plan's partial-output workspace C[M,N] (bf16) to a
+ * device buffer `dst` on `stream` (for checking the producer by itself).
+ */
+int entwine_read_partial(entwine_plan_t plan, void* dst, void* stream);
+
+/*
+ * entwine_plan_export - write one of the plan's integer tables to host memory.
+ *   what      ENTWINE_EXPORT_*
+ *   host_buf  host pointer, or NULL to query the size only
+ *   bytes     in: capacity of host_buf; out: bytes needed / written
+ * Errors: ENTWINE_ERR_INVALID (unknown table, or capacity too small: *bytes is still set).
+ */
+int entwine_plan_export(entwine_plan_t plan, int what, void* host_buf, size_t* bytes);
+
+/*
+ * entwine_last_status - synchronise the stream of the plan's last launch and read its
+ * status block into out[8]:
+ *   0 code (ENTWINE_OK / ENTWINE_ERR_TIMEOUT / ENTWINE_ERR_INTERNAL), 1 CTA that reported,
+ *   2 task or block it was on, 3 flags published, 4 tiles reduced, 5 tiles pushed,
+ *   6 T_G: ns from the first CTA's start to the last producer block's completion (Eq. 3),
+ *   7 T_end: ns from the first CTA's start to the last CTA's exit (end-to-end, Sec. 3.2).
+ * Returns out[0].  Clears the pending status.
+ */
+int entwine_last_status(entwine_plan_t plan, int64_t out[8]);
+
+/* entwine_destroy - free the plan and everything it owns (synchronises its last stream). */
+int entwine_destroy(entwine_plan_t plan);
+
+/* entwine_strerror - static, human-readable text for a return code. */
+const char* entwine_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENTWINE_H_ */
