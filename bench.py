@@ -1,0 +1,466 @@
+#!/usr/bin/env python
+"""Benchmark of the fused GEMM-ReduceScatter hot path (one-rank emulation on one B200).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one entwine_gemm_rs call (schedule already planned; GEMM + per-tile flags + scatter
+push + reduction in one launch) over one batch of seeded synthetic input.  The headline value
+is 2*M*N*K_local / device time, with inputs resident in HBM and the L2 flushed between timed
+steps.  One JSON line is printed on stdout by rank 0.
+
+With --gpus N > 1 (under torchrun) every rank runs an independent replica of the same problem
+on its own GPU (the path does not shard: "replicas only"); no data-path collective is issued.
+
+--impl reference times the CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused GEMM-RS TFLOP/s and fraction of max(tensor peak, HBM) roofline"
+# Peaks measured on this machine (used only if MEASURED_PEAKS.json is absent).
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic (bytes read + written per launch) of the fused kernel from an ncu capture of
+# the named workload; see profiles/.  None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+# Launch configuration per workload: communication SMs, tile order.
+LAUNCH = {
+    "attn_out_proj": dict(n_comm_sms=20, order=1, rank=1),
+    "mlp_down_proj": dict(n_comm_sms=20, order=1, rank=5),
+    "short_k_comm_bound": dict(n_comm_sms=16, order=1, rank=2),
+    "tiny": dict(n_comm_sms=4, order=1, rank=0),
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def roofline_seconds(wl, peaks):
+    t_tc = wl.flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = wl.comm_bytes / (peaks["hbm_gbs"] * 1e9)
+    return t_tc, t_hbm
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def lines(self):
+        try:
+            return sum(1 for _ in open(self.path))
+        except Exception:
+            return 0
+
+    def wait_for_samples(self, n, timeout_s=10.0):
+        t0 = time.perf_counter()
+        while self.proc is not None and self.lines() < n and time.perf_counter() - t0 < timeout_s:
+            time.sleep(0.02)
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def _dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), \
+        int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def run_cpu_oracle(wl, launch, rows_per_pass, passes):
+    """Times the oracle (float64 GEMM of the sampled rows + reduce-scatter definition + the
+    whole integer schedule) and returns (best seconds, flops of one pass, threads used)."""
+    import numpy as np
+    import torch
+    from oracle import entwine_oracle as O
+    from paper_2609_11562_b200 import inputs as I
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    r = launch["rank"]
+    x = launch["n_comm_sms"] or 148
+    full = rows_per_pass >= wl.M
+    rows = None if full else np.linspace(0, wl.M - 1, rows_per_pass).astype(np.int64)
+    times = []
+    for _ in range(passes):
+        t0 = time.perf_counter()
+        O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, launch["order"], x, rows=rows)
+        times.append(time.perf_counter() - t0)
+    n_rows = wl.M if full else rows_per_pass
+    return times, 2.0 * n_rows * wl.N * wl.K, torch.get_num_threads()
+
+
+def main_reference(args, wl, launch):
+    rank, _, world = _dist_env()
+    if rank != 0:
+        return 0
+    # size the per-step sample so that the whole run stays within a couple of minutes
+    probe, flops_probe, threads = run_cpu_oracle(wl, launch, min(256, wl.M), 1)
+    sec_per_row = probe[0] / min(256, wl.M)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rows = int(max(128, min(wl.M, (budget / max(sec_per_row, 1e-9)) // 128 * 128)))
+    times, flops, threads = run_cpu_oracle(wl, launch, rows, args.steps + args.warmup)
+    timed = times[args.warmup:]
+    mean = sum(timed) / len(timed)
+    value = flops / mean / 1e12
+    sample = (f"{rows} of {wl.M} rows of the float64 partial GEMM and its magnitude sums + the full "
+              f"integer schedule per step" + (" + reduce-scatter definition" if rows >= wl.M else ""))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K,
+                   "tile_order": "interleaved" if launch["order"] else "row_major"},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def time_steps(fn, steps, warmup, flush, torch):
+    """Device time of `steps` calls of fn with the L2 flushed before each; returns µs list."""
+    for _ in range(warmup):
+        flush.zero_()
+        fn()
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(steps):
+        flush.zero_()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) * 1e3 for a, b in evs]
+
+
+def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
+    """All device-side numbers of one workload on the current device."""
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+    res = {}
+    us = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), steps, warmup, flush, torch)
+    st = plan.last_status()
+    res["fused_us"] = us
+    res["status"] = st
+    if detailed:
+        # the producer alone (uncontended GEMM time) and the consumer alone
+        res["gemm_only_us"] = time_steps(lambda: plan.gemm_only(A, Bm), max(5, steps // 4), 3, flush, torch)
+        plan.last_status()
+        res["comm_only_us"] = time_steps(lambda: plan.comm_only(None, P, out, send, 0), max(5, steps // 4), 3,
+                                         flush, torch)
+        plan.last_status()
+        # unfused sequence: library GEMM into a bf16 [M,N] buffer, then reduce + scatter on all SMs
+        Cfull = torch.empty(wl.M, wl.N, dtype=torch.bfloat16, device="cuda")
+        plan0 = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], 0, rank=launch["rank"])
+
+        def unfused():
+            torch.matmul(A, Bm.t(), out=Cfull)
+            plan0.comm_only(Cfull, P, out, send, 0)
+        res["unfused_us"] = time_steps(unfused, max(5, steps // 4), 3, flush, torch)
+        plan0.last_status()
+        res["cublas_gemm_us"] = time_steps(lambda: torch.matmul(A, Bm.t(), out=Cfull), max(5, steps // 4), 3,
+                                           flush, torch)
+        plan0.destroy()
+        del Cfull
+    plan.destroy()
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="attn_out_proj")
+    ap.add_argument("--impl", default="entwine", choices=["entwine", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and comparisons")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", default=None, choices=["fused", "gemm", "comm"],
+                    help="profiling aid: run warmup+steps launches of one mode on the workload and exit")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "entwine" else args.warmup
+
+    from paper_2609_11562_b200 import inputs as I
+    wl = I.CONFIGS[args.workload]
+    launch = LAUNCH[args.workload]
+    if args.impl == "reference":
+        return main_reference(args, wl, launch)
+
+    import torch
+    rank, local_rank, world = _dist_env()
+    if not torch.cuda.is_available():
+        print("bench.py needs a CUDA device (there is no CPU fallback)", file=sys.stderr)
+        return 2
+    torch.cuda.set_device(local_rank % torch.cuda.device_count())
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    from paper_2609_11562_b200 import build as B
+    if rank == 0:
+        B.build()
+    if dist is not None:
+        dist.barrier()
+    from paper_2609_11562_b200 import entwine as E
+
+    peaks = load_peaks()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB of L2
+    if args.kernel_only:
+        A, Bm = I.make_operands(wl, device="cuda")
+        P = I.make_peer_partials(wl, device="cuda")
+        out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+        plan.gemm_only(A, Bm)
+        fn = {"fused": lambda: plan.gemm_rs(A, Bm, P, out, send), "gemm": lambda: plan.gemm_only(A, Bm),
+              "comm": lambda: plan.comm_only(None, P, out, send, 0)}[args.kernel_only]
+        us = time_steps(fn, args.steps, args.warmup, flush, torch)
+        plan.last_status()
+        print(json.dumps({"kernel_only": args.kernel_only, "workload": wl.name,
+                          "median_us": statistics.median(us)}))
+        plan.destroy()
+        return 0
+    dev_uuid = "GPU-" + str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+    sampler = ClockSampler(dev_uuid)
+
+    # ---- headline: timed region of exactly `steps` fused calls -------------------------------
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+    sampler.start()
+    for _ in range(args.warmup):
+        flush.zero_()
+        plan.gemm_rs(A, Bm, P, out, send)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    lines_before = sampler.lines()
+    t_wall0 = time.perf_counter()
+    evs = []
+    for _ in range(args.steps):
+        flush.zero_()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        plan.gemm_rs(A, Bm, P, out, send)
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t_wall0
+    # A short timed region can end before nvidia-smi's next sample: keep the same load running,
+    # untimed, until two samples under load exist.
+    extended = False
+    t_ext = time.perf_counter()
+    while sampler.proc is not None and sampler.lines() < lines_before + 2 and time.perf_counter() - t_ext < 5.0:
+        extended = True
+        for _ in range(20):
+            flush.zero_()
+            plan.gemm_rs(A, Bm, P, out, send)
+        torch.cuda.synchronize()
+    clocks = sampler.stop()
+    clocks["sampled"] = ("during the timed region" if not extended else
+                         "timed region shorter than the sampling period: same load continued untimed")
+    us = [a.elapsed_time(b) * 1e3 for a, b in evs]
+    status = plan.last_status()
+    total_us = sum(us)
+    if dist is not None:
+        t = torch.tensor([total_us], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_us = float(t.item())
+    mean_us = total_us / args.steps
+    value = world * wl.flops / (mean_us * 1e-6) / 1e12
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------
+    hA, hB, hP = A.cpu().pin_memory(), Bm.cpu().pin_memory(), P.cpu().pin_memory()
+    hOut = torch.empty(wl.R, wl.N, dtype=torch.bfloat16).pin_memory()
+    hSend = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        plan.gemm_rs_host(hA, hB, hP, hOut, hSend)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        plan.gemm_rs_host(hA, hB, hP, hOut, hSend)
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    h2d = (wl.M * wl.K + wl.N * wl.K + (wl.W - 1) * wl.R * wl.N) * 2
+    d2h = (wl.R * wl.N + (wl.W - 1) * wl.R * wl.N) * 2
+    e2e = {"value": world * wl.flops / e2e_s / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3}
+    plan.destroy()
+    del hA, hB, hP, hOut, hSend, A, Bm, P, out, send
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant (only) kernel of a step --------------------------------------
+    t_tc, t_hbm = roofline_seconds(wl, peaks)
+    tensor_bound = t_tc >= t_hbm
+    if tensor_bound:
+        achieved = wl.flops / (mean_us * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"]}
+    else:
+        achieved = wl.comm_bytes / (mean_us * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"]}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
+    roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
+    roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
+    roof["kernel"] = "entwine_fused_kernel<256>"
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": mean_us / 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K,
+                   "n_comm_sms": launch["n_comm_sms"],
+                   "tile_order": "interleaved" if launch["order"] else "row_major", "block": "128x256",
+                   "emulated_rank": launch["rank"], "l2": "flushed between timed steps (512 MiB memset)",
+                   "multi_gpu": "replicas only"},
+        "us_per_call": {"mean": mean_us, "median": statistics.median(us), "min": min(us)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roof,
+        "device_status": {"t_gemm_us": status["t_gemm_ns"] / 1e3, "t_end_us": status["t_end_ns"] / 1e3,
+                          "tail_us": (status["t_end_ns"] - status["t_gemm_ns"]) / 1e3},
+        "wall_s_timed_region": wall,
+    }
+
+    # ---- comparisons and the other LLM-shaped configurations -----------------------------------
+    if not args.no_extra:
+        extra = {}
+        names = [wl.name] + [n for n in ("attn_out_proj", "mlp_down_proj", "short_k_comm_bound") if n != wl.name]
+        for name in names:
+            w2 = I.CONFIGS[name]
+            r = measure_workload(w2, LAUNCH[name], max(10, args.steps // 2), 5, flush, torch, E, I, True)
+            med = statistics.median
+            fused = med(r["fused_us"])
+            tc, hb = roofline_seconds(w2, peaks)
+            e = {
+                "fused_us": fused, "fused_tflops": w2.flops / fused / 1e6,
+                "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
+                "bound": "tensor" if tc >= hb else "hbm",
+                "unfused_cublas_then_reduce_us": med(r["unfused_us"]),
+                "speedup_vs_unfused": med(r["unfused_us"]) / fused,
+                "cublas_gemm_us": med(r["cublas_gemm_us"]),
+                "gemm_alone_us": med(r["gemm_only_us"]),
+                "comm_alone_all_sms_us": med(r["comm_only_us"]),
+                "comm_alone_GBps": w2.comm_bytes / med(r["comm_only_us"]) / 1e3,
+                "overlap_efficiency": med(r["gemm_only_us"]) / fused,
+                "tail_us": (r["status"]["t_end_ns"] - r["status"]["t_gemm_ns"]) / 1e3,
+                "n_comm_sms": LAUNCH[name]["n_comm_sms"],
+            }
+            # Eq. 4 generalised to the emulation's push + reduce bytes, from the measured window
+            t_g = r["status"]["t_gemm_ns"] * 1e-9
+            if t_g > 0:
+                e["b_req_GBps"] = w2.comm_bytes / t_g / 1e9
+                e["b_measured_GBps"] = w2.comm_bytes / (r["status"]["t_end_ns"] * 1e-9) / 1e9
+            extra[name] = e
+        line["comparisons"] = extra
+
+    # ---- CPU baseline: the oracle on the host cores --------------------------------------------
+    if not args.no_cpu_baseline:
+        rows = wl.M if wl.flops <= 5e10 else 512
+        probe, _, _ = run_cpu_oracle(wl, launch, rows, 1)
+        passes = int(max(3, min(40, 12.0 / max(probe[0], 1e-3))))
+        times, flops, threads = run_cpu_oracle(wl, launch, rows, passes)
+        line["cpu_baseline"] = {
+            "value": flops / min(times) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
+            "sample": (f"{rows} of {wl.M} rows of the float64 partial GEMM and its magnitude sums"
+                       + (" + reduce-scatter definition" if rows >= wl.M else "") +
+                       f" + the full integer schedule, best of {passes} passes ({sum(times):.1f} s in total)")}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

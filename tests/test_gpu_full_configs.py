@@ -1,0 +1,111 @@
+"""Full-size parity for the LLM-shaped configurations, in the launch configuration the
+benchmark times.  The oracle computes sampled rows one by one (float64); properties that
+hold at any size cover every element: pushed tiles are bit-identical to the stored partial,
+the reduction is the order-exact fp32 sum of the stored contributions, counts are exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import entwine_oracle as O
+from paper_2609_11562_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2609_11562_b200 import build as B
+    B.build()
+    from paper_2609_11562_b200 import entwine as E
+
+# (workload, rank, orders, budgets): the budgets are the ones the configurations name
+FULL = [
+    (I.ATTN_OUT, 1, (1, 0), (20,)),
+    (I.MLP_DOWN, 5, (1,), (20,)),
+    (I.SHORT_K, 2, (1, 0), (8, 16, 24)),
+]
+
+
+def _rows_to_f64(t, rows):
+    return O.bf16_bits_to_f64(I.bits(t[rows]))
+
+
+@pytest.mark.parametrize("wl,r,orders,budgets", FULL, ids=lambda v: getattr(v, "name", None))
+def test_full_size_sampled_parity(wl, r, orders, budgets):
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    R, W = wl.R, wl.W
+    rng = np.random.default_rng(wl.seed)
+    # sampled rows of the M x N partial: a band in every partition incl. first / last rows
+    rows = np.unique(np.concatenate(
+        [np.array([d * R, d * R + R - 1]) for d in range(W)] +
+        [rng.integers(0, wl.M, 48)] + [r * R + rng.integers(0, R, 48)]))
+    Ab, Bb = I.bits(A[rows]), I.bits(Bm)
+    C_rows = O.partial_gemm(Ab, Bb)           # float64, rows x N
+    S_rows = O.abs_gemm(Ab, Bb)
+    own = (rows >= r * R) & (rows < (r + 1) * R)
+    own_rows = rows[own]
+    peers_rows = np.stack([_rows_to_f64(P[q], own_rows) for q in range(W - 1)])
+    ref_out = C_rows[own] + peers_rows.sum(0)
+    S_out = S_rows[own] + np.abs(peers_rows).sum(0)
+    for order in orders:
+        for n_comm in budgets:
+            p = E.Plan(wl.M, wl.N, wl.K, W, order, n_comm, rank=r)
+            c = p.counts()
+            out = torch.full((R, wl.N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            send = torch.full((W - 1, R, wl.N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            p.gemm_rs(A, Bm, P, out, send)
+            st = p.last_status()
+            assert st["flags_published"] == c["flags_published"] == W * c["Q"]
+            assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+            # sampled rows against the float64 oracle
+            got_out = _rows_to_f64(out, own_rows - r * R)
+            err = np.abs(got_out - ref_out)
+            tol = O.tolerance(ref_out, S_out)
+            assert (err <= tol).all(), f"out worst err/tol {np.max(err / tol):.3f}"
+            for i, row in enumerate(rows):
+                d = int(row // R)
+                if d == r:
+                    continue
+                got = O.bf16_bits_to_f64(I.bits(send[O.peer_slot(d, r), row - d * R]))
+                e = np.abs(got - C_rows[i])
+                assert (e <= O.tolerance(C_rows[i], S_rows[i])).all()
+            # every element: copies are exact, the reduction is the fp32 rank-order sum
+            Cd = torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device="cuda")
+            p.read_partial(Cd)
+            torch.cuda.synchronize()
+            for slot, d in enumerate(dd for dd in range(W) if dd != r):
+                assert torch.equal(send[slot], Cd[d * R:(d + 1) * R])
+            acc = Cd[r * R:(r + 1) * R].float()
+            for q in range(W - 1):
+                acc = acc + P[q, r * R:(r + 1) * R].float()
+            assert torch.equal(out, acc.to(torch.bfloat16))
+            assert not torch.isnan(out.float()).any()
+            del Cd, acc, out, send
+            p.destroy()
+
+
+def test_sweep_corner_shapes_smoke_parity():
+    """Two corners of the sweep grid (smallest and a large one), both orders, budget 0 and 32:
+    exact counts and the any-size properties."""
+    for wl in (I.sweep_workloads()[0], I.sweep_workloads()[-4]):
+        A, Bm = I.make_operands(wl, device="cuda")
+        P = I.make_peer_partials(wl, device="cuda")
+        R, W, r = wl.R, wl.W, wl.W - 1
+        for order, n_comm in ((0, 0), (1, 32)):
+            p = E.Plan(wl.M, wl.N, wl.K, W, order, n_comm, rank=r)
+            out = torch.empty((R, wl.N), dtype=torch.bfloat16, device="cuda")
+            send = torch.empty((W - 1, R, wl.N), dtype=torch.bfloat16, device="cuda")
+            p.gemm_rs(A, Bm, P, out, send)
+            st = p.last_status()
+            c = p.counts()
+            assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+            Cd = torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device="cuda")
+            p.read_partial(Cd)
+            ref = torch.matmul(A, Bm.t())          # library GEMM as a whole-matrix sanity check
+            assert (Cd.float() - ref.float()).abs().max() <= 0.02 * ref.float().abs().max()
+            for slot, d in enumerate(dd for dd in range(W) if dd != r):
+                assert torch.equal(send[slot], Cd[d * R:(d + 1) * R])
+            acc = Cd[r * R:(r + 1) * R].float()
+            for q in range(W - 1):
+                acc = acc + P[q, r * R:(r + 1) * R].float()
+            assert torch.equal(out, acc.to(torch.bfloat16))
+            p.destroy()
