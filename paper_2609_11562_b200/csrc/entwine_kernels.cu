@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 
@@ -19,10 +20,16 @@ namespace entwine {
 constexpr int kBM = 128;          // producer block rows = reduction tile rows
 constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes = one swizzle row)
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
-constexpr int kThreads = 256;     // warp 0: TMA, warp 1: MMA + TMEM owner, warps 4-7: epilogue
+constexpr int kThreads = 320;     // producer: warp 0 TMA, warp 1 MMA + TMEM owner, warps 4-7 epilogue
+                                  // consumer: warp 0 polls flags + issues TMA loads, warps 1-8
+                                  // reduce, warp 9 issues the TMA stores
 constexpr int kEpiWarp0 = 4;
 constexpr int kEpiThreads = 128;
+constexpr int kConsThreads = 256;
+constexpr int kStoreWarp = 9;
 constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abort flag
+constexpr int kMaxSlots = 8;          // consumer ring depth (upper bound)
+constexpr int kEpiStageBytes = 8192;  // per epilogue warp: 32 rows x 128 columns of bf16
 
 template <int BN>
 struct Cfg {
@@ -30,10 +37,20 @@ struct Cfg {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kPipeBytes = kStages * kStageBytes;
   static constexpr int kTmemCols = 2 * BN;  // two accumulators: epilogue overlaps next mainloop
-  static constexpr int kBarBytes = 256;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes + 1024;  // + align slack
 };
+// Shared-memory map (offsets from a 1024-byte aligned base), identical for both block widths:
+//   [0, 196608)        producer: TMA/MMA operand ring          | consumer: tile ring
+//   [196608, 229376)   producer: epilogue staging (4 x 8 KiB)  | consumer: tile ring (cont.)
+//   [229376, 229888)   mbarriers + TMEM base slot
+constexpr int kPipeBytes = 196608;
+constexpr int kStagingOff = kPipeBytes;
+constexpr int kRingBytes = kPipeBytes + 4 * kEpiStageBytes;
+constexpr int kBarOff = kRingBytes;
+constexpr int kBarBytes = 512;
+constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
+static_assert(Cfg<256>::kPipeBytes == kPipeBytes && Cfg<128>::kPipeBytes == kPipeBytes, "smem map");
 
 struct KParams {
   // geometry
@@ -47,14 +64,14 @@ struct KParams {
   int mode;       // Mode
   int help;       // producers / finished consumers take tasks from other lists
   int skip_wait;  // treat every flag as published (consumer in isolation)
+  int rs;         // rows of a tile moved per reduce step (all W contributions of those rows)
+  int prs;        // rows of a tile moved per push step
+  int slot_bytes; // bytes of one consumer ring slot
+  int n_slots;    // consumer ring depth
   unsigned epoch;  // flag value of this producer run
   unsigned seq;    // launch counter: selects the status slot
   unsigned long long wait_budget_ns;
   // memory
-  __nv_bfloat16* C;              // partial output workspace [M,N] (or caller's partial)
-  const __nv_bfloat16* peers;    // [W-1][M][N]
-  __nv_bfloat16* out;            // [R][N]
-  __nv_bfloat16* send;           // [W-1][R][N]
   unsigned* flags_own;           // [W][Q]
   const unsigned* flags_peer;    // [W-1][Q]
   const Task* tasks;
@@ -62,6 +79,17 @@ struct KParams {
   int* list_head;                // [x]
   StatusSlot* status;            // [2]
   unsigned* done_ctr;
+};
+
+// Tensor maps of one launch.  Loads of A and B and the epilogue's stores of C use the
+// 128-byte swizzle; the consumer's maps are plain row-major boxes of 128 columns x rs rows.
+struct KMaps {
+  CUtensorMap a, b;      // operands
+  CUtensorMap c_st;      // partial C, box 64 x 32, swizzled (epilogue stores)
+  CUtensorMap c_ld;      // partial C as the consumer reads it
+  CUtensorMap p_ld;      // incoming partials viewed as [(W-1)*M, N]
+  CUtensorMap out_st;    // out_shard [R, N]
+  CUtensorMap send_st;   // send_bufs viewed as [(W-1)*R, N]
 };
 
 // ------------------------------------------------------------------------------------------
@@ -104,6 +132,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {  // <= N groups still reading shared memory
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_done() {  // <= N groups not yet complete
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void fence_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem),
                "r"(cols)
@@ -162,6 +208,15 @@ __device__ __forceinline__ void st_release_gpu(unsigned* p, unsigned v) {
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, const uint4& v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64
 // elements) written by TMA with 128-byte swizzle: 8-row groups are 1024 bytes apart.
@@ -183,11 +238,14 @@ __device__ __forceinline__ constexpr uint32_t instr_desc() {
 // ------------------------------------------------------------------------------------------
 // status helpers
 // ------------------------------------------------------------------------------------------
+struct SlotMeta {
+  int kind;      // 0 reduce step, 1 push tile, -1 end of work
+  int dst_x;     // column of the destination box
+  int dst_y;     // row of the destination box in the destination map
+};
 struct CtaShared {
-  volatile int abort;   // another role of this CTA (or a peer CTA) gave up
-  int claim;            // broadcast of the claimed task index
-  int wait_ok;          // broadcast of the flag wait's result
-  uint32_t tmem_base;
+  volatile int abort;   // a role of this CTA (or another CTA) gave up
+  SlotMeta meta[kMaxSlots];
 };
 
 __device__ __forceinline__ void report(const KParams& P, int code, long long where) {
@@ -216,7 +274,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const K
   }
 }
 
-// Bounded acquire-poll of one flag (Sec. 4.2: thread 0 polls with acquire loads).
+// Bounded acquire-poll of one flag (Sec. 4.2: acquire loads until the flag is published).
 __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
   if (ld_acquire_gpu(f) >= P.epoch) return true;
   unsigned long long t0 = 0;
@@ -228,12 +286,12 @@ __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
       if (t0 == 0) t0 = now;
       else if (now - t0 > P.wait_budget_ns) return false;
     }
-    __nanosleep(40);
+    __nanosleep(32);
   }
 }
 
 // ------------------------------------------------------------------------------------------
-// consumer: ReduceTile and the scatter push (Sec. 4.2)
+// consumer: flag polling, scatter push and ReduceTile (Sec. 4.2) as a TMA ring pipeline
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& v) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -253,128 +311,238 @@ __device__ __forceinline__ uint4 pack_bf16x8(const float (&a)[8]) {
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-constexpr int kChunksPerTile = kTile * kTile * 2 / 16;  // 16-byte chunks in a 128x128 bf16 tile
-
-// out = bf16( fp32(own) + sum over peers in ascending rank order ), one writer per element.
-template <int NP>
-__device__ __forceinline__ void reduce_tile(const __nv_bfloat16* own, const __nv_bfloat16* peer0,
-                                            long long peer_stride, __nv_bfloat16* dst, long long N,
-                                            int n_peers_rt) {
-  constexpr int U = (NP > 0 && NP <= 3) ? 4 : 2;
-  const int n_peers = NP > 0 ? NP : n_peers_rt;
-  for (int it = 0; it < kChunksPerTile / kThreads; it += U) {
-    uint4 o[U];
-    uint4 pv[U][NP > 0 ? NP : 1];
-    long long off[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int idx = threadIdx.x + (it + u) * kThreads;
-      off[u] = (long long)(idx >> 4) * N + (idx & 15) * 8;
-      o[u] = __ldcg(reinterpret_cast<const uint4*>(own + off[u]));
-      if (NP > 0) {
-#pragma unroll
-        for (int q = 0; q < (NP > 0 ? NP : 1); ++q)
-          pv[u][q] = __ldcs(reinterpret_cast<const uint4*>(peer0 + q * peer_stride + off[u]));
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      acc_bf16x8(a, o[u]);  // start from the local contribution
-      if (NP > 0) {
-#pragma unroll
-        for (int q = 0; q < (NP > 0 ? NP : 1); ++q) acc_bf16x8(a, pv[u][q]);
-      } else {
-        for (int q = 0; q < n_peers; ++q)
-          acc_bf16x8(a, __ldcs(reinterpret_cast<const uint4*>(peer0 + q * peer_stride + off[u])));
-      }
-      __stcs(reinterpret_cast<uint4*>(dst + off[u]), pack_bf16x8(a));
-    }
-  }
-}
-
-__device__ __forceinline__ void push_tile(const __nv_bfloat16* src, __nv_bfloat16* dst, long long N) {
-  constexpr int U = 8;
-  static_assert(kChunksPerTile / kThreads == U, "one pass");
-  uint4 v[U];
-  long long off[U];
-#pragma unroll
-  for (int u = 0; u < U; ++u) {
-    const int idx = threadIdx.x + u * kThreads;
-    off[u] = (long long)(idx >> 4) * N + (idx & 15) * 8;
-    v[u] = __ldcg(reinterpret_cast<const uint4*>(src + off[u]));
-  }
-#pragma unroll
-  for (int u = 0; u < U; ++u) __stcs(reinterpret_cast<uint4*>(dst + off[u]), v[u]);
-}
-
 struct CommCounters {
   unsigned reduced = 0, pushed = 0;
 };
 
-// Walk consumer lists starting at `first_list`; every task is claimed through its list's
-// head counter, so a list is always consumed in order (Sec. 3.1) whoever executes it.
-__device__ void consumer_walk(const KParams& P, CtaShared* sh, int first_list, int n_lists_to_visit,
-                              CommCounters* cnt) {
-  const long long MN = (long long)P.M * P.N;
-  const long long RN = P.R * (long long)P.N;
-  for (int li = 0; li < n_lists_to_visit; ++li) {
-    int j = first_list + li;
-    if (j >= P.x) j -= P.x;
-    const int base = P.list_offs[j];
-    const int len = P.list_offs[j + 1] - base;
-    for (;;) {
-      if (threadIdx.x == 0) {
-        // cheap look before the atomic so that exhausted lists cost one load
-        int head = *reinterpret_cast<volatile int*>(&P.list_head[j]);
-        sh->claim = (head >= len) ? len : atomicAdd(&P.list_head[j], 1);
+// One CTA's consumer work: warp 0 claims tasks from `n_lists` consumer lists starting at
+// `first_list` (each list is consumed in order through its head counter, Sec. 3.1), polls
+// the tile flags with one lane per contributing rank, and streams the tiles through a ring
+// of shared-memory slots with TMA; warps 1-8 reduce the slots and warp 9 stores them.
+__device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
+                                  int first_list, int n_lists, CommCounters* cnt) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t ring_bar = smem_base + kBarOff + 256;
+  auto full_bar = [&](int s) { return ring_bar + 8u * s; };
+  auto empty_bar = [&](int s) { return ring_bar + 8u * (kMaxSlots + s); };
+  auto red_bar = [&](int s) { return ring_bar + 8u * (2 * kMaxSlots + s); };
+  const int rs = P.rs;
+  const int sub_bytes = rs * kTile * 2;      // one source's rows of one step
+  const int n_sub = kTile / rs;
+
+  if (warp == 0) {
+    // ---------------- claim, poll, load ----------------
+    int it = 0;
+    bool ok = true;
+    const long long MN = (long long)P.M * P.N, RN = P.R * (long long)P.N;
+    // Drains list j: claims go through the list's head counter, so the list is consumed in
+    // order whoever executes it.  The next claim is issued before the current task is
+    // processed, which hides the atomic's latency.
+    auto drain = [&](int j) {
+      const int base = P.list_offs[j];
+      const int len = P.list_offs[j + 1] - base;
+      // two claims are kept in flight so that the atomics' latency is hidden
+      int c0 = len, c1 = len;
+      if (lane == 0) {
+        c0 = atomicAdd(&P.list_head[j], 1);
+        c1 = atomicAdd(&P.list_head[j], 1);
       }
-      __syncthreads();
-      const int i = sh->claim;
-      __syncthreads();
-      if (i >= len) break;
-      const Task task = P.tasks[base + i];
-      // index check: record and skip instead of touching memory out of range
-      bool bad = task.src_off < 0 || task.src_off + (long long)(kTile - 1) * P.N + kTile > MN ||
-                 task.dst_off < 0 || task.dst_off + (long long)(kTile - 1) * P.N + kTile > RN ||
-                 task.t < 0 || task.t >= P.Q || task.d < 0 || task.d >= P.W ||
-                 (task.kind == 1 && (task.slot < 0 || task.slot >= P.W - 1));
-      if (bad) {
-        if (threadIdx.x == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
-        continue;
-      }
-      if (!P.skip_wait) {
-        if (threadIdx.x == 0) {
-          // local flag first, then the peers in ascending rank order (Sec. 4.2)
-          bool ok = wait_flag(&P.flags_own[task.d * P.Q + task.t], P);
-          if (ok && task.kind == 0) {
-            for (int q = 0; ok && q < P.W - 1; ++q) ok = wait_flag(&P.flags_peer[q * P.Q + task.t], P);
+      // window of 32 task records, one per lane, refilled when a claim falls outside it
+      int win = -(1 << 30);
+      Task mine;
+      mine.kind = 0; mine.d = 0; mine.t = 0; mine.slot = 0; mine.src_off = 0; mine.dst_off = 0;
+      while (ok) {
+        const int i = __shfl_sync(0xffffffffu, c0, 0);
+        if (i >= len) break;
+        c0 = c1;
+        if (lane == 0) c1 = atomicAdd(&P.list_head[j], 1);
+        if (i < win || i >= win + 32) {
+          win = i;
+          mine = P.tasks[base + min(i + lane, len - 1)];
+        }
+        const int src = i - win;
+        Task task;
+        task.kind = __shfl_sync(0xffffffffu, mine.kind, src);
+        task.d = __shfl_sync(0xffffffffu, mine.d, src);
+        task.t = __shfl_sync(0xffffffffu, mine.t, src);
+        task.slot = __shfl_sync(0xffffffffu, mine.slot, src);
+        task.src_off = __shfl_sync(0xffffffffu, mine.src_off, src);
+        task.dst_off = __shfl_sync(0xffffffffu, mine.dst_off, src);
+        // index check: record and skip instead of touching memory out of range
+        const bool bad = task.src_off < 0 || task.src_off + (long long)(kTile - 1) * P.N + kTile > MN ||
+                         task.dst_off < 0 || task.dst_off + (long long)(kTile - 1) * P.N + kTile > RN ||
+                         task.t < 0 || task.t >= P.Q || task.d < 0 || task.d >= P.W ||
+                         (task.kind == 1 && (task.slot < 0 || task.slot >= P.W - 1));
+        if (bad) {
+          if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
+          continue;
+        }
+        if (!P.skip_wait) {
+          // lane 0 polls the local flag, lanes 1.. the peers' flags in rank order (Sec. 4.2);
+          // the warp proceeds when all W contributions of the tile are published
+          bool mine_ok = true;
+          if (lane == 0) mine_ok = wait_flag(&P.flags_own[task.d * P.Q + task.t], P);
+          else if (task.kind == 0) {
+            for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
+              mine_ok = wait_flag(&P.flags_peer[q * P.Q + task.t], P);
           }
-          if (!ok) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
-          sh->wait_ok = ok ? 1 : 0;
+          ok = __all_sync(0xffffffffu, mine_ok);
+          if (!ok) {
+            if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
+            break;
+          }
+          fence_async_all();  // the TMA reads below are ordered after the acquires
         }
-        __syncthreads();  // extends thread 0's acquire to the whole CTA (Sec. 4.2)
-        const int ok = sh->wait_ok;
-        __syncthreads();
-        if (!ok) return;
-      }
-      const __nv_bfloat16* src = P.C + task.src_off;
-      if (task.kind == 0) {
-        const __nv_bfloat16* peer0 = P.peers + task.src_off;
-        __nv_bfloat16* dst = P.out + task.dst_off;
-        switch (P.W - 1) {
-          case 1: reduce_tile<1>(src, peer0, MN, dst, P.N, 1); break;
-          case 3: reduce_tile<3>(src, peer0, MN, dst, P.N, 3); break;
-          case 7: reduce_tile<7>(src, peer0, MN, dst, P.N, 7); break;
-          default: reduce_tile<0>(src, peer0, MN, dst, P.N, P.W - 1); break;
+        const int trow = task.t / P.nTn, tcol = task.t % P.nTn;
+        const int col = tcol * kTile;
+        const int src_row = task.d * (int)P.R + trow * kTile;  // row of the tile in an [M,N] buffer
+        if (task.kind == 0) {
+          // one step = rs rows of all W contributions; lane q issues contribution q's load
+          for (int sub = 0; ok && sub < n_sub; ++sub, ++it) {
+            const int slot = it % P.n_slots;
+            const uint32_t ph = (it / P.n_slots) & 1;
+            bool free_slot = true;
+            if (lane == 0) {
+              free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
+              if (free_slot) {
+                sh->meta[slot].kind = 0;
+                sh->meta[slot].dst_x = col;
+                sh->meta[slot].dst_y = trow * kTile + sub * rs;
+                mbar_arrive_expect_tx(full_bar(slot), P.W * sub_bytes);
+              }
+            }
+            ok = __all_sync(0xffffffffu, free_slot);
+            if (!ok) break;
+            const uint32_t dst = smem_base + slot * P.slot_bytes;
+            // the local contribution first, then the peers in ascending rank order
+            for (int q = lane; q < P.W; q += 32) {
+              if (q == 0) tma_load_2d(dst, &maps.c_ld, col, src_row + sub * rs, full_bar(slot));
+              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld, col, (q - 1) * P.M + src_row + sub * rs, full_bar(slot));
+            }
+          }
+          if (lane == 0) cnt->reduced++;
+        } else {
+          for (int r0 = 0; ok && r0 < kTile; r0 += P.prs, ++it) {
+            const int slot = it % P.n_slots;
+            const uint32_t ph = (it / P.n_slots) & 1;
+            bool free_slot = true;
+            if (lane == 0) {
+              free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
+              if (free_slot) {
+                sh->meta[slot].kind = 1;
+                sh->meta[slot].dst_x = col;
+                sh->meta[slot].dst_y = task.slot * (int)P.R + trow * kTile + r0;
+                mbar_arrive_expect_tx(full_bar(slot), P.prs * kTile * 2);
+              }
+            }
+            ok = __all_sync(0xffffffffu, free_slot);
+            if (!ok) break;
+            const uint32_t dst = smem_base + slot * P.slot_bytes;
+            for (int rr = lane * rs; rr < P.prs; rr += 32 * rs)
+              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld, col, src_row + r0 + rr, full_bar(slot));
+          }
+          if (lane == 0) cnt->pushed++;
         }
-        if (threadIdx.x == 0) cnt->reduced++;
-      } else {
-        push_tile(src, P.send + (long long)task.slot * RN + task.dst_off, P.N);
-        if (threadIdx.x == 0) cnt->pushed++;
+        if (!ok && lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
       }
+    };
+    // the CTA's own list first
+    if (n_lists > 0) drain(first_list);
+    // then the other lists: every lane looks at one list per round, lists with work are drained
+    while (ok && n_lists > 1) {
+      bool any = false;
+      for (int j0 = 0; ok && j0 < P.x; j0 += 32) {
+        int j = first_list + 1 + j0 + lane;  // walk starts after the own list
+        const bool in = j0 + lane < P.x - 1;
+        while (j >= P.x) j -= P.x;
+        bool work = false;
+        if (in) work = *reinterpret_cast<volatile int*>(&P.list_head[j]) < P.list_offs[j + 1] - P.list_offs[j];
+        unsigned mask = __ballot_sync(0xffffffffu, work);
+        while (ok && mask) {
+          const int b = __ffs(mask) - 1;
+          mask &= mask - 1;
+          int jj = first_list + 1 + j0 + b;
+          while (jj >= P.x) jj -= P.x;
+          any = true;
+          drain(jj);
+        }
+      }
+      if (!any) break;
     }
+    // end-of-work marker so that the reducing warps leave their loop
+    if (lane == 0) {
+      const int slot = it % P.n_slots;
+      const uint32_t ph = (it / P.n_slots) & 1;
+      const bool free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
+      if (!free_slot) sh->abort = 1;
+      sh->meta[slot].kind = -1;
+      mbar_arrive(full_bar(slot));
+    }
+    __syncwarp();
+  } else if (warp <= kConsThreads / 32) {
+    // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
+    const int ctid = threadIdx.x - 32;
+    for (int it = 0;; ++it) {
+      const int slot = it % P.n_slots;
+      const uint32_t ph = (it / P.n_slots) & 1;
+      if (!mbar_wait(full_bar(slot), ph, P, sh)) {
+        sh->abort = 1;
+        break;
+      }
+      const int kind = sh->meta[slot].kind;
+      if (kind < 0) break;
+      if (kind == 0) {
+        const uint32_t sbase = smem_base + slot * P.slot_bytes;
+        // start from the local contribution, add the peers in ascending rank order, fp32
+        for (int c = ctid; c < rs * (kTile * 2 / 16); c += kConsThreads) {
+          float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          const uint32_t addr = sbase + c * 16;
+          acc_bf16x8(a, ld_shared_v4(addr));
+#pragma unroll 4
+          for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
+          st_shared_v4(addr, pack_bf16x8(a));  // in place over the local contribution's rows
+        }
+        fence_async_smem();  // generic-proxy writes above -> visible to the TMA store
+      }
+      // one arrival per warp hands the slot to the store warp (a push step is forwarded by the
+      // store warp alone; the arrival then only says that this warp has read the slot's header)
+      __syncwarp();
+      if (lane == 0) mbar_arrive(red_bar(slot));
+    }
+  } else if (warp == kStoreWarp && lane == 0) {
+    // ---------------- store the slots, recycle them ----------------
+    int prev_slot = -1;
+    for (int it = 0;; ++it) {
+      const int slot = it % P.n_slots;
+      const uint32_t ph = (it / P.n_slots) & 1;
+      if (!mbar_wait(full_bar(slot), ph, P, sh)) {
+        sh->abort = 1;
+        break;
+      }
+      const int kind = sh->meta[slot].kind;
+      if (kind < 0) break;
+      const int dst_x = sh->meta[slot].dst_x, dst_y = sh->meta[slot].dst_y;
+      const uint32_t sbase = smem_base + slot * P.slot_bytes;
+      if (!mbar_wait(red_bar(slot), ph, P, sh)) {
+        sh->abort = 1;
+        break;
+      }
+      if (kind == 0) {
+        tma_store_2d(&maps.out_st, dst_x, dst_y, sbase);
+      } else {
+        for (int rr = 0; rr < P.prs; rr += rs) tma_store_2d(&maps.send_st, dst_x, dst_y + rr, sbase + rr * kTile * 2);
+      }
+      bulk_commit();
+      // the previous slot is free once its store has finished reading shared memory
+      if (prev_slot >= 0) {
+        bulk_wait_read<1>();
+        mbar_arrive(empty_bar(prev_slot));
+      }
+      prev_slot = slot;
+    }
+    bulk_wait_done<0>();  // every store of this CTA is complete before it exits
   }
+  __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -382,39 +550,27 @@ __device__ void consumer_walk(const KParams& P, CtaShared* sh, int first_list, i
 // ------------------------------------------------------------------------------------------
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
-entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
-                     const __grid_constant__ CUtensorMap tmap_b, const KParams P) {
+entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   __shared__ CtaShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   StatusSlot* st = &P.status[P.seq & 1];
-
-  if (threadIdx.x == 0) {
-    sh.abort = 0;
-    sh.claim = 0;
-    sh.wait_ok = 0;
-    sh.tmem_base = 0;
-    atomicMin(&st->t_start, globaltimer_ns());
-  }
-  CommCounters cnt;
-  unsigned published = 0;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t smem_base = smem_u32(smem);
+  const uint32_t bar_base = smem_base + kBarOff;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + 2 + a); };
+  const uint32_t tmem_slot = bar_base + 8u * (2 * C::kStages + 4);
   const bool is_producer = (int)blockIdx.x >= P.n_ded && P.mode != MODE_COMM_ONLY;
   const int g = (int)blockIdx.x - P.n_ded;
 
-  if (is_producer) {
-    // ---------------- producer: tcgen05 GEMM over blocks p = g, g+G, ... ----------------
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                               ~uintptr_t(1023));
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t bar_base = smem_base + C::kStages * C::kStageBytes;
-    auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
-    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
-    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + 2 + a); };
-    const uint32_t tmem_slot = bar_base + 8u * (2 * C::kStages + 4);
-
-    if (threadIdx.x == 0) {
+  if (threadIdx.x == 0) {
+    sh.abort = 0;
+    atomicMin(&st->t_start, globaltimer_ns());
+    if (is_producer) {
       for (int s = 0; s < C::kStages; ++s) {
         mbar_init(full_bar(s), 1);
         mbar_init(empty_bar(s), 1);
@@ -423,14 +579,24 @@ entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
         mbar_init(tfull_bar(a), 1);
         mbar_init(tempty_bar(a), kEpiThreads / 32);
       }
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int s = 0; s < kMaxSlots; ++s) {  // consumer ring: full, empty, reduced
+      mbar_init(bar_base + 256 + 8u * s, 1);
+      mbar_init(bar_base + 256 + 8u * (kMaxSlots + s), 1);
+      mbar_init(bar_base + 256 + 8u * (2 * kMaxSlots + s), kConsThreads / 32);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  CommCounters cnt;
+  unsigned published = 0;
+
+  if (is_producer) {
+    // ---------------- producer: tcgen05 GEMM over blocks p = g, g+G, ... ----------------
     if (warp == 1) tmem_alloc(tmem_slot, C::kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base =
-        *reinterpret_cast<volatile uint32_t*>(smem + C::kStages * C::kStageBytes + 8 * (2 * C::kStages + 4));
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + kBarOff + 8 * (2 * C::kStages + 4));
     const int KB = (P.K + kBK - 1) / kBK;
     const int n_my = (g < P.P_blk) ? (P.P_blk - g + P.G - 1) / P.G : 0;
 
@@ -449,8 +615,8 @@ entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
           if (!mbar_wait(empty_bar(stage), phase ^ 1, P, &sh)) { ok = false; break; }
           mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
           const uint32_t a_dst = smem_base + stage * C::kStageBytes;
-          tma_load_2d(a_dst, &tmap_a, kb * kBK, mb * kBM, full_bar(stage));
-          tma_load_2d(a_dst + C::kABytes, &tmap_b, kb * kBK, nb * BN, full_bar(stage));
+          tma_load_2d(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage));
+          tma_load_2d(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage));
           if (++stage == C::kStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -486,9 +652,11 @@ entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -2); }
-    } else if (warp >= kEpiWarp0) {
-      // ---- epilogue: TMEM -> bf16 -> partial C, then publish the block's tile flags ----
-      const int q = warp & 3;  // TMEM lane quarter this warp may read
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiThreads / 32) {
+      // ---- epilogue: TMEM -> bf16 -> swizzled staging -> TMA store of the partial C, then the
+      //      block's tile flags ----
+      const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
+      const uint32_t stg = smem_base + kStagingOff + q * kEpiStageBytes;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
@@ -503,29 +671,49 @@ entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
         ok = __all_sync(0xffffffffu, ok);  // reconverge; the warp leaves the loop together
         if (!ok) break;
         tc_fence_after();
-        const long long row = (long long)mb * kBM + q * 32 + lane;
-        __nv_bfloat16* crow = P.C + row * P.N + (long long)nb * BN;
         const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + acc * BN;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(taddr + c * 32, v);
-          tmem_ld_wait();
-          uint4 o[4];
-          uint32_t* ow = reinterpret_cast<uint32_t*>(o);
+        for (int h = 0; h < BN / kTile; ++h) {
+          // one 128-column reduction tile: 32 rows x 256 bytes per warp, as two swizzled boxes
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1]));
-            ow[e] = *reinterpret_cast<uint32_t*>(&h);
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(taddr + h * kTile + cc * 32, v);
+            tmem_ld_wait();
+            if (h == BN / kTile - 1 && cc == 3) {
+              // last read of this accumulator: the MMA warp may overwrite it
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(tempty_bar(acc));
+            }
+            const uint32_t box = stg + (cc >> 1) * 4096 + lane * 128;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              uint4 o;
+              uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * e + 2 * u]),
+                                                          __uint_as_float(v[8 * e + 2 * u + 1]));
+                ow[u] = *reinterpret_cast<uint32_t*>(&hh);
+              }
+              const int chunk = (cc & 1) * 4 + e;  // 16-byte chunk inside the 128-byte row
+              st_shared_v4(box + ((chunk ^ (lane & 7)) << 4), o);
+            }
           }
-          uint4* dstp = reinterpret_cast<uint4*>(crow + c * 32);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) dstp[e] = o[e];
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            const int x0 = nb * BN + h * kTile, y0 = mb * kBM + q * 32;
+            tma_store_2d(&maps.c_st, x0, y0, stg);
+            tma_store_2d(&maps.c_st, x0 + 64, y0, stg + 4096);
+            bulk_commit();
+            if (h == BN / kTile - 1) bulk_wait_done<0>();  // stores complete: publishable
+            else bulk_wait_read<0>();                      // staging may be rewritten
+          }
+          __syncwarp();
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));  // accumulator may be overwritten
-        // all of the block's stores, then the flags (Sec. 4.2)
+        // all of the block's stores (of all four warps), then the flags (Sec. 4.2)
         named_bar_sync(1, kEpiThreads);
         if (warp == kEpiWarp0 && lane == 0) {
           for (int c = 0; c < P.cpb; ++c) {
@@ -548,28 +736,30 @@ entwine_fused_kernel(const __grid_constant__ CUtensorMap tmap_a,
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
     __syncthreads();
+  } else {
+    __syncthreads();  // barrier initialisation visible to the whole CTA
   }
 
   // ---------------- consumer ----------------
   if (P.mode != MODE_GEMM_ONLY && !sh.abort) {
+    int first = 0, count = 0;
     if (!is_producer) {
       // dedicated consumer block j: its own list, then (shared-pool analogue) the others
-      const int j = (int)blockIdx.x % P.x;
-      const bool owns = (int)blockIdx.x < P.x;
-      if (owns) consumer_walk(P, &sh, j, 1, &cnt);
-      if (P.help || !owns) consumer_walk(P, &sh, owns ? (j + 1) % P.x : j, owns ? P.x - 1 : P.x, &cnt);
+      first = (int)blockIdx.x % P.x;
+      count = ((int)blockIdx.x < P.x && !P.help) ? 1 : P.x;
     } else if (P.n_ded == 0) {
       // non-overlapped use of all SMs: block g consumes list g (then helps)
-      if (g < P.x) consumer_walk(P, &sh, g, 1, &cnt);
-      if (P.help) consumer_walk(P, &sh, (g + 1) % P.x, P.x - 1, &cnt);
+      first = g % P.x;
+      count = P.help ? P.x : (g < P.x ? 1 : 0);
     } else if (P.help) {
-      consumer_walk(P, &sh, g % P.x, P.x, &cnt);
+      first = g % P.x;
+      count = P.x;
     }
+    if (count > 0) consumer_pipeline(P, maps, &sh, smem_base, first, count, &cnt);
   }
 
   // ---------------- exit bookkeeping ----------------
   __syncthreads();
-  // the epilogue's publishing thread adds its own count
   if (is_producer && warp == kEpiWarp0 && lane == 0 && published)
     atomicAdd(&st->flags_published, (unsigned long long)published);
   __syncthreads();
@@ -636,17 +826,20 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D map over a row-major bf16 matrix [rows, cols] with a (box_rows x 64-column) box and
-// 128-byte swizzle; out-of-range elements read as zero (K tails).
-static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+// 2-D map over a row-major bf16 matrix [rows, cols] with a (box_rows x box_cols) box;
+// out-of-range elements read as zero (K tails).  `swizzle128` selects the 128-byte swizzle
+// (box_cols must then be 64 elements = 128 bytes).
+static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols,
+                     int box_rows, bool swizzle128) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
   cuuint64_t strides[1] = {cuuint64_t(cols) * 2};
-  cuuint32_t box[2] = {cuuint32_t(kBK), cuuint32_t(box_rows)};
+  cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
   cuuint32_t estr[2] = {1, 1};
   CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS;
 }
@@ -748,19 +941,17 @@ void device_release(Plan* p) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int BN>
-static int launch_bn(Plan* p, const KParams& kp, const CUtensorMap& ma, const CUtensorMap& mb, int grid,
-                     cudaStream_t stream) {
-  using C = Cfg<BN>;
+static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
   static bool configured = false;
   auto kern = entwine_fused_kernel<BN>;
   if (!configured) {
-    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     int per_sm = 0;
-    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, C::kSmemBytes));
+    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
     if (per_sm < 1) return ENTWINE_ERR_RESOURCES;
     configured = true;
   }
-  kern<<<grid, kThreads, C::kSmemBytes, stream>>>(ma, mb, kp);
+  kern<<<grid, kThreads, kSmemBytes, stream>>>(maps, kp);
   CK(cudaGetLastError());
   return ENTWINE_OK;
 }
@@ -817,11 +1008,19 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   d->seq += 1;
   kp.seq = d->seq;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  kp.C = (mode == MODE_COMM_ONLY && partial) ? const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(partial))
-                                             : d->C;
-  kp.peers = static_cast<const __nv_bfloat16*>(peers);
-  kp.out = static_cast<__nv_bfloat16*>(out);
-  kp.send = static_cast<__nv_bfloat16*>(send);
+  // consumer ring: a reduce step moves rs rows of all W contributions (about 32 KiB), a push
+  // step moves as many rows of one tile as fit in the same slot
+  int rs = 64;
+  while (rs > 1 && int64_t(g.W) * rs * kTile * 2 > 32768) rs /= 2;
+  int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
+  int prs = rs;
+  while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
+  slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
+  if (slot_bytes * 2 > kRingBytes) return ENTWINE_ERR_RESOURCES;
+  kp.rs = rs;
+  kp.prs = prs;
+  kp.slot_bytes = slot_bytes;
+  kp.n_slots = std::min(kMaxSlots, kRingBytes / slot_bytes);
   kp.flags_own = d->flags_own;
   kp.flags_peer = d->flags_peer;
   kp.tasks = d->tasks;
@@ -848,13 +1047,24 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
     if (grid < p->x) kp.help = 1;
   }
 
-  CUtensorMap ma, mb;
-  std::memset(&ma, 0, sizeof(ma));
-  std::memset(&mb, 0, sizeof(mb));
-  if (mode != MODE_COMM_ONLY) {
-    if (!make_map(&ma, A, g.M, g.K, kBM) || !make_map(&mb, B, g.N, g.K, g.BN)) return ENTWINE_ERR_CUDA;
-  }
-  rc = (g.BN == 256) ? launch_bn<256>(p, kp, ma, mb, grid, stream) : launch_bn<128>(p, kp, ma, mb, grid, stream);
+  KMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  const void* c_src = (mode == MODE_COMM_ONLY && partial) ? partial : d->C;
+  // maps of buffers a mode does not touch point at the workspace so that they stay encodable
+  const void* a_p = (mode != MODE_COMM_ONLY) ? A : d->C;
+  const void* b_p = (mode != MODE_COMM_ONLY) ? B : d->C;
+  const bool comm = mode != MODE_GEMM_ONLY;
+  bool ok = make_map(&maps.a, a_p, (mode != MODE_COMM_ONLY) ? g.M : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
+                     kBK, kBM, true) &&
+            make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
+                     kBK, (mode != MODE_COMM_ONLY) ? g.BN : kBM, true) &&
+            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.c_ld, c_src, g.M, g.N, kTile, rs, false) &&
+            make_map(&maps.p_ld, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, rs, false) &&
+            make_map(&maps.out_st, comm ? out : d->C, comm ? g.R : g.M, g.N, kTile, rs, false) &&
+            make_map(&maps.send_st, comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, rs, false);
+  if (!ok) return ENTWINE_ERR_CUDA;
+  rc = (g.BN == 256) ? launch_bn<256>(p, kp, maps, grid, stream) : launch_bn<128>(p, kp, maps, grid, stream);
   if (rc != ENTWINE_OK) return rc;
   p->launched = true;
   d->last_stream = stream;
