@@ -74,8 +74,12 @@ enum {
   ENTWINE_OPT_NUM_SMS         = 6, /* [pre] override the SM count used for planning (testing
                                       without a device; default: the device's SM count, 148 if
                                       there is no device)                                        */
-  ENTWINE_OPT_POISON_PARTIAL  = 7  /* 1: fill the partial-output workspace with NaN patterns
+  ENTWINE_OPT_POISON_PARTIAL  = 7, /* 1: fill the partial-output workspace with NaN patterns
                                       before each launch (ordering stress test; default 0)       */
+  ENTWINE_OPT_PAIR_CTAS       = 8  /* [pre] 1 (default): where the order allows it, two CTAs of a
+                                      cluster compute a 256x256 pair tile (tcgen05 cta_group::2:
+                                      two producer blocks that share a block column, each CTA
+                                      loading half of the B panel); 0: every CTA works alone     */
 };
 
 /* What entwine_plan_export can write.  Integer tables, host memory, for bit-exact diffs. */

@@ -74,6 +74,8 @@ struct Plan {
   int num_sms = 148;
   bool num_sms_overridden = false;
   int tail_help = 1;
+  int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles
+  bool pair = false;        // pair tiles in use for this plan
   int poison = 0;
   int64_t wait_budget_ns = 2000000000LL;
   int64_t withhold_peer = -1;

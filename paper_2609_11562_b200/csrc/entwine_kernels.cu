@@ -31,12 +31,17 @@ constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abor
 constexpr int kMaxSlots = 8;          // consumer ring depth (upper bound)
 constexpr int kEpiStageBytes = 8192;  // per epilogue warp: 32 rows x 128 columns of bf16
 
-template <int BN>
+// PAIR = two CTAs of a cluster compute a 256 x 256 pair tile with tcgen05 cta_group::2: each
+// CTA loads its own 128 rows of A and half (128 rows) of the B panel, so a CTA moves 32 KiB
+// per k-block instead of 48 KiB.
+template <int BN, bool PAIR>
 struct Cfg {
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static_assert(!PAIR || BN == 256, "pair tiles are 256 wide");
+  static constexpr int kBRows = PAIR ? 128 : BN;  // rows of B this CTA loads per stage
   static constexpr int kABytes = kBM * kBK * 2;
-  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kBBytes = kBRows * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = 196608 / kStageBytes;  // 4 (128x256), 6 (128x128 or pair)
   static constexpr int kPipeBytes = kStages * kStageBytes;
   static constexpr int kTmemCols = 2 * BN;  // two accumulators: epilogue overlaps next mainloop
 };
@@ -50,7 +55,8 @@ constexpr int kRingBytes = kPipeBytes + 4 * kEpiStageBytes;
 constexpr int kBarOff = kRingBytes;
 constexpr int kBarBytes = 512;
 constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
-static_assert(Cfg<256>::kPipeBytes == kPipeBytes && Cfg<128>::kPipeBytes == kPipeBytes, "smem map");
+static_assert(Cfg<256, false>::kPipeBytes == kPipeBytes && Cfg<128, false>::kPipeBytes == kPipeBytes &&
+                  Cfg<256, true>::kPipeBytes == kPipeBytes && Cfg<256, true>::kStages <= 8, "smem map");
 
 struct KParams {
   // geometry
@@ -58,8 +64,8 @@ struct KParams {
   int rowsT, nBn, nTn, Lb, P_blk, Q, cpb;
   long long R;
   // launch shape
-  int n_ded;      // CTAs [0, n_ded) are dedicated consumers
-  int G;          // CTAs [n_ded, n_ded+G) are producers
+  int G;          // CTAs [0, G) are producers (pairs of them in pair mode)
+  int n_ded;      // CTAs [G, G + n_ded) are dedicated consumers
   int x;          // consumer lists
   int mode;       // Mode
   int help;       // producers / finished consumers take tasks from other lists
@@ -150,6 +156,60 @@ __device__ __forceinline__ void fence_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void fence_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load of a CTA pair: the bytes are counted on the barrier at `bar_cluster_addr`, which may
+// live in the peer CTA (no multicast: each CTA fetches its own box).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem),
+               "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+               : "memory");
+}
+// commit of a CTA pair's MMAs, arriving on the barrier at the same offset in both CTAs
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((unsigned short)3)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem),
                "r"(cols)
@@ -230,9 +290,21 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   return d;
 }
 // Instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, M = 128.
-template <int BN>
+template <int BN, int MM>
 __device__ __forceinline__ constexpr uint32_t instr_desc() {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(kBM >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(MM >> 4) << 24);
+}
+
+// Producer block handled by CTA `rank` of the pair that works on pair index u.  Both blocks of
+// a pair share the block column (the B panel).  Interleaved order (W even): positions 2u and
+// 2u+1 of Eq. 1, i.e. two destinations at once.  Row-major order (even tile rows per
+// partition): vertically adjacent blocks of one partition.
+__device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) {
+  if (P.order == ENTWINE_ORDER_INTERLEAVED) return 2 * u + rank;
+  const int half = P.Lb / 2;
+  const int d = u / half, rem = u - d * half;
+  const int v = rem / P.nBn, nb = rem - v * P.nBn;
+  return d * P.Lb + (2 * v + rank) * P.nBn + nb;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -548,10 +620,10 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
 // ------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------
-template <int BN>
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, PAIR>;
   extern __shared__ uint8_t smem_raw[];
   __shared__ CtaShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -564,8 +636,11 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + 2 + a); };
   const uint32_t tmem_slot = bar_base + 8u * (2 * C::kStages + 4);
-  const bool is_producer = (int)blockIdx.x >= P.n_ded && P.mode != MODE_COMM_ONLY;
-  const int g = (int)blockIdx.x - P.n_ded;
+  const bool is_producer = (int)blockIdx.x < P.G && P.mode != MODE_COMM_ONLY;
+  const int g = (int)blockIdx.x;                 // producer index
+  const int cidx = (int)blockIdx.x - P.G;        // consumer index of a dedicated consumer CTA
+  const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+  const bool leader = cta_rank == 0;
 
   if (threadIdx.x == 0) {
     sh.abort = 0;
@@ -577,7 +652,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       }
       for (int a = 0; a < 2; ++a) {
         mbar_init(tfull_bar(a), 1);
-        mbar_init(tempty_bar(a), kEpiThreads / 32);
+        mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * (kEpiThreads / 32));
       }
     }
     for (int s = 0; s < kMaxSlots; ++s) {  // consumer ring: full, empty, reduced
@@ -591,43 +666,63 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   unsigned published = 0;
 
   if (is_producer) {
-    // ---------------- producer: tcgen05 GEMM over blocks p = g, g+G, ... ----------------
-    if (warp == 1) tmem_alloc(tmem_slot, C::kTmemCols);
+    // ---------------- producer: tcgen05 GEMM ----------------
+    if (warp == 1) {
+      if (PAIR) tmem_alloc_pair(tmem_slot, C::kTmemCols);
+      else tmem_alloc(tmem_slot, C::kTmemCols);
+    }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + kBarOff + 8 * (2 * C::kStages + 4));
     const int KB = (P.K + kBK - 1) / kBK;
-    const int n_my = (g < P.P_blk) ? (P.P_blk - g + P.G - 1) / P.G : 0;
+    // work units: blocks p = g, g+G, ... or, for pairs, pair indices u = g/2, g/2 + G/2, ...
+    const int n_units = PAIR ? P.P_blk / 2 : P.P_blk;
+    const int unit0 = PAIR ? g / 2 : g;
+    const int stride = PAIR ? P.G / 2 : P.G;
+    const int n_my = (unit0 < n_units) ? (n_units - unit0 + stride - 1) / stride : 0;
+    auto block_of = [&](int i, int* d, int* l) {
+      const int unit = unit0 + i * stride;
+      const int p = PAIR ? pair_position(P, unit, (int)cta_rank) : unit;
+      if (P.order == ENTWINE_ORDER_INTERLEAVED) { *d = p % P.W; *l = p / P.W; }
+      else { *d = p / P.Lb; *l = p - *d * P.Lb; }
+    };
 
     if (warp == 0 && lane == 0) {
-      // ---- TMA producer ----
+      // ---- TMA producer (every CTA loads its own operands) ----
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int i = 0; ok && i < n_my; ++i) {
-        const int p = g + i * P.G;
         int d, l;
-        if (P.order == ENTWINE_ORDER_INTERLEAVED) { d = p % P.W; l = p / P.W; }
-        else { d = p / P.Lb; l = p - d * P.Lb; }
+        block_of(i, &d, &l);
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
         for (int kb = 0; kb < KB; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, P, &sh)) { ok = false; break; }
-          mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
           const uint32_t a_dst = smem_base + stage * C::kStageBytes;
-          tma_load_2d(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage));
-          tma_load_2d(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage));
+          if (PAIR) {
+            // both CTAs' bytes are counted on the leader's barrier, which the leader arms
+            if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * C::kStageBytes);
+            const uint32_t lead_bar = map_to_cta(full_bar(stage), 0);
+            tma_load_2d_pair(a_dst, &maps.a, kb * kBK, mb * kBM, lead_bar);
+            tma_load_2d_pair(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN + (int)cta_rank * C::kBRows, lead_bar);
+          } else {
+            mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
+            tma_load_2d(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage));
+            tma_load_2d(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage));
+          }
           if (++stage == C::kStages) { stage = 0; phase ^= 1; }
         }
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -1); }
-    } else if (warp == 1 && lane == 0) {
-      // ---- MMA issuer ----
+    } else if (warp == 1 && lane == 0 && leader) {
+      // ---- MMA issuer (the leader CTA issues for the pair) ----
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
-      constexpr uint32_t idesc = instr_desc<BN>();
+      constexpr uint32_t idesc = instr_desc<BN, PAIR ? 256 : 128>();
       bool ok = true;
       for (int i = 0; ok && i < n_my; ++i) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh)) { ok = false; break; }
@@ -642,13 +737,17 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // advancing K by 16 elements = 32 bytes = 2 descriptor address units
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
           }
-          tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if (PAIR) tc_commit_pair(empty_bar(stage));
+          else tc_commit(empty_bar(stage));
           if (++stage == C::kStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));  // accumulator complete
+        if (PAIR) tc_commit_pair(tfull_bar(acc));  // accumulator complete (both CTAs' halves)
+        else tc_commit(tfull_bar(acc));
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -2); }
@@ -661,10 +760,8 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int i = 0; ok && i < n_my; ++i) {
-        const int p = g + i * P.G;
         int d, l;
-        if (P.order == ENTWINE_ORDER_INTERLEAVED) { d = p % P.W; l = p / P.W; }
-        else { d = p / P.Lb; l = p - d * P.Lb; }
+        block_of(i, &d, &l);
         const int trow = l / P.nBn, nb = l % P.nBn;
         const int mb = d * P.rowsT + trow;
         ok = mbar_wait(tfull_bar(acc), acc_phase, P, &sh);
@@ -684,7 +781,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
               // last read of this accumulator: the MMA warp may overwrite it
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(tempty_bar(acc));
+              if (lane == 0) {
+                if (leader) mbar_arrive(tempty_bar(acc));
+                else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+              }
             }
             const uint32_t box = stg + (cc >> 1) * 4096 + lane * 128;
 #pragma unroll
@@ -733,8 +833,13 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       const unsigned long long t0 = globaltimer_ns();
       while (globaltimer_ns() - t0 < 200000ULL) __nanosleep(1000);
     }
+    // the peer may still read this CTA's operands / signal its barriers until it is done too
+    if (PAIR) cluster_sync_all();
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, C::kTmemCols);
+    if (warp == 1) {
+      if (PAIR) tmem_dealloc_pair(tmem_base, C::kTmemCols);
+      else tmem_dealloc(tmem_base, C::kTmemCols);
+    }
     __syncthreads();
   } else {
     __syncthreads();  // barrier initialisation visible to the whole CTA
@@ -745,8 +850,8 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     int first = 0, count = 0;
     if (!is_producer) {
       // dedicated consumer block j: its own list, then (shared-pool analogue) the others
-      first = (int)blockIdx.x % P.x;
-      count = ((int)blockIdx.x < P.x && !P.help) ? 1 : P.x;
+      first = cidx % P.x;
+      count = (cidx < P.x && !P.help) ? 1 : P.x;
     } else if (P.n_ded == 0) {
       // non-overlapped use of all SMs: block g consumes list g (then helps)
       first = g % P.x;
@@ -940,18 +1045,38 @@ void device_release(Plan* p) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-template <int BN>
+template <int BN, bool PAIR>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
   static bool configured = false;
-  auto kern = entwine_fused_kernel<BN>;
+  auto kern = entwine_fused_kernel<BN, PAIR>;
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(unsigned(grid), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (!configured) {
     CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     int per_sm = 0;
     CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
     if (per_sm < 1) return ENTWINE_ERR_RESOURCES;
+    if (PAIR) {
+      // every cluster of the grid must be resident at once: producers and consumers wait on
+      // each other inside one launch
+      int clusters = 0;
+      CK(cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg));
+      if (clusters * 2 < grid) return ENTWINE_ERR_RESOURCES;
+    }
     configured = true;
   }
-  kern<<<grid, kThreads, kSmemBytes, stream>>>(maps, kp);
+  CK(cudaLaunchKernelEx(&cfg, kern, maps, kp));
   CK(cudaGetLastError());
   return ENTWINE_OK;
 }
@@ -1030,14 +1155,15 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.done_ctr = d->done_ctr;
 
   int grid;
+  const bool pair = p->pair;
   if (mode == MODE_FUSED) {
     kp.n_ded = p->n_comm_ctas;
     kp.G = p->n_gemm_ctas;
     grid = p->n_comm_ctas + p->n_gemm_ctas;
   } else if (mode == MODE_GEMM_ONLY) {
     kp.n_ded = 0;
-    kp.G = p->num_sms;
-    grid = p->num_sms;
+    kp.G = pair ? (p->num_sms & ~1) : p->num_sms;
+    grid = kp.G;
   } else {
     grid = (n_ctas <= 0) ? p->num_sms : n_ctas;
     if (grid > p->num_sms) return ENTWINE_ERR_INVALID;
@@ -1045,6 +1171,13 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
     kp.G = 0;
     // with fewer CTAs than lists the CTAs must visit every list
     if (grid < p->x) kp.help = 1;
+  }
+  // a cluster launch needs whole clusters: an odd grid gets one more consumer CTA, which owns
+  // no list and only helps
+  if (pair && (grid & 1)) {
+    if (grid + 1 > p->num_sms) grid -= 1, kp.n_ded -= 1;
+    else grid += 1, kp.n_ded += 1;
+    if (kp.n_ded < p->x) kp.help = 1;
   }
 
   KMaps maps;
@@ -1057,14 +1190,16 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   bool ok = make_map(&maps.a, a_p, (mode != MODE_COMM_ONLY) ? g.M : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
                      kBK, kBM, true) &&
             make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
-                     kBK, (mode != MODE_COMM_ONLY) ? g.BN : kBM, true) &&
+                     kBK, (mode != MODE_COMM_ONLY) ? (pair ? 128 : g.BN) : kBM, true) &&
             make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true) &&
             make_map(&maps.c_ld, c_src, g.M, g.N, kTile, rs, false) &&
             make_map(&maps.p_ld, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, rs, false) &&
             make_map(&maps.out_st, comm ? out : d->C, comm ? g.R : g.M, g.N, kTile, rs, false) &&
             make_map(&maps.send_st, comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, rs, false);
   if (!ok) return ENTWINE_ERR_CUDA;
-  rc = (g.BN == 256) ? launch_bn<256>(p, kp, maps, grid, stream) : launch_bn<128>(p, kp, maps, grid, stream);
+  if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
+  else if (g.BN == 256) rc = launch_bn<256, false>(p, kp, maps, grid, stream);
+  else rc = launch_bn<128, false>(p, kp, maps, grid, stream);
   if (rc != ENTWINE_OK) return rc;
   p->launched = true;
   d->last_stream = stream;

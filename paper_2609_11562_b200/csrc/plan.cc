@@ -146,14 +146,23 @@ int finalize_plan(Plan* p) {
   }
   if (p->n_comm_sms < 0 || p->n_comm_sms >= p->num_sms) return ENTWINE_ERR_INVALID;
   if (p->rank < 0 || p->rank >= p->g.W) return ENTWINE_ERR_INVALID;
+  // CTA-pair producer tiles need two blocks that share a block column: positions 2u, 2u+1 of
+  // the interleaved order (W even) or vertically adjacent blocks of a partition (row-major,
+  // even number of tile rows per partition).
+  const Geometry& g = p->g;
+  p->pair = p->pair_opt && g.BN == 256 && p->num_sms >= 2 &&
+            ((p->order == ENTWINE_ORDER_INTERLEAVED && g.W % 2 == 0) ||
+             (p->order == ENTWINE_ORDER_ROW_MAJOR && g.rowsT % 2 == 0));
   if (p->n_comm_sms == 0) {
     // non-overlapped use of all SMs: every CTA produces, then consumes
     p->n_comm_ctas = 0;
-    p->n_gemm_ctas = p->num_sms;
-    p->x = p->num_sms;
+    p->n_gemm_ctas = p->pair ? (p->num_sms & ~1) : p->num_sms;
+    p->x = p->n_gemm_ctas;
   } else {
     p->n_comm_ctas = p->n_comm_sms;
     p->n_gemm_ctas = p->num_sms - p->n_comm_sms;
+    if (p->pair) p->n_gemm_ctas &= ~1;
+    if (p->n_gemm_ctas < 1) return ENTWINE_ERR_INVALID;
     p->x = p->n_comm_sms;
   }
   build_tables(p->g, p->order, p->rank, p->x, p->n_gemm_ctas, p->n_comm_ctas, &p->tables);
@@ -239,6 +248,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       }
       return rc;
     }
+    case ENTWINE_OPT_PAIR_CTAS:
+      if (p->launched || (value != 0 && value != 1)) return ENTWINE_ERR_INVALID;
+      p->pair_opt = int(value);
+      return entwine::finalize_plan(p);
     case ENTWINE_OPT_POISON_PARTIAL:
       if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
       p->poison = int(value);

@@ -23,7 +23,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 ORDER_ROW_MAJOR, ORDER_INTERLEAVED = 0, 1
 OK, ERR_INVALID, ERR_RESOURCES, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
 OPT_RANK, OPT_BLOCK_N, OPT_WAIT_BUDGET_NS, OPT_TAIL_HELP = 1, 2, 3, 4
-OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL = 5, 6, 7
+OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL, OPT_PAIR_CTAS = 5, 6, 7, 8
 (EXPORT_COUNTS, EXPORT_ORDER, EXPORT_TILES, EXPORT_FLAG_SEQ, EXPORT_LIST_OFFS, EXPORT_TASKS,
  EXPORT_PEER_OFFS) = range(7)
 
@@ -98,7 +98,8 @@ class Plan:
         self.tile_order, self.n_comm_sms = tile_order, n_comm_sms
         self.rank = 0
         keys = {"rank": OPT_RANK, "block_n": OPT_BLOCK_N, "wait_budget_ns": OPT_WAIT_BUDGET_NS,
-                "tail_help": OPT_TAIL_HELP, "num_sms": OPT_NUM_SMS, "poison_partial": OPT_POISON_PARTIAL}
+                "tail_help": OPT_TAIL_HELP, "num_sms": OPT_NUM_SMS, "poison_partial": OPT_POISON_PARTIAL,
+                "pair_ctas": OPT_PAIR_CTAS}
         # num_sms first: it bounds the others
         for name in sorted(options, key=lambda n: n != "num_sms"):
             self.set_option(keys[name], options[name])

@@ -102,10 +102,10 @@ def test_producer_alone_matches_oracle_gemm(wl):
     C_ref = O.partial_gemm(I.bits(A), I.bits(Bm))
     S = O.abs_gemm(I.bits(A), I.bits(Bm))
     Ad, Bd = A.cuda(), Bm.cuda()
-    for order, BN in itertools.product((E.ORDER_ROW_MAJOR, E.ORDER_INTERLEAVED), (128, 256)):
-        if wl.N % BN:
+    for order, BN, pair in itertools.product((E.ORDER_ROW_MAJOR, E.ORDER_INTERLEAVED), (128, 256), (0, 1)):
+        if wl.N % BN or (pair and BN == 128):
             continue
-        p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, 0, block_n=BN)
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, 0, block_n=BN, pair_ctas=pair)
         Cd = torch.full((wl.M, wl.N), float("nan"), dtype=torch.bfloat16, device="cuda")
         p.gemm_only(Ad, Bd)
         p.read_partial(Cd)
@@ -163,10 +163,10 @@ def test_fused_matches_oracle(wl):
     ranks = range(wl.W) if wl.W <= 2 else (0, wl.W - 1)
     for r in ranks:
         res = None
-        for order, BN, n_comm in itertools.product((0, 1), (128, 256), budgets):
-            if wl.N % BN:
+        for order, BN, n_comm, pair in itertools.product((0, 1), (128, 256), budgets, (0, 1)):
+            if wl.N % BN or (pair and BN == 128):
                 continue
-            p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, block_n=BN, rank=r)
+            p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, block_n=BN, rank=r, pair_ctas=pair)
             c = p.counts()
             if res is None:
                 res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, BN, order, c["x"])
