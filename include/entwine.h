@@ -55,7 +55,8 @@ enum {
   ENTWINE_ERR_RESOURCES = -2, /* not enough SMs / shared memory for a co-resident launch     */
   ENTWINE_ERR_CUDA      = -3, /* a CUDA call failed, or there is no CUDA device              */
   ENTWINE_ERR_TIMEOUT   = -4, /* a device-side wait ran out of its budget                    */
-  ENTWINE_ERR_INTERNAL  = -5  /* a device-side index check failed                            */
+  ENTWINE_ERR_INTERNAL  = -5, /* a device-side index check failed                            */
+  ENTWINE_ERR_TOO_LARGE = -6  /* the problem does not fit entwine_gemm_rs_static's fixed scratch */
 };
 
 /* Option keys for entwine_set_option. Options marked [pre] must be set before the first
@@ -191,6 +192,43 @@ int entwine_plan_export(entwine_plan_t plan, int what, void* host_buf, size_t* b
  * Returns out[0].  Clears the pending status.
  */
 int entwine_last_status(entwine_plan_t plan, int64_t out[8]);
+
+/*
+ * entwine_gemm_rs_static - entwine_gemm_rs for callers that must not allocate.  (The paper
+ * has no counterpart; this entry point exists for the library's users only.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unaffordable - inside
+ * a region that an application has declared allocation-free (a serving loop with a frozen
+ * memory plan, a real-time path where cudaMalloc's implicit device synchronisation or its
+ * latency is unacceptable), or a host that has handed all device memory to another
+ * allocator and has nothing left for cudaMalloc to give.  entwine_gemm_rs allocates its
+ * workspace with cudaMalloc at a plan's first launch; this variant never calls cudaMalloc,
+ * cudaFree or any allocating routine.
+ *
+ * Instead of plan-owned memory it uses one fixed array inside the library image (9 MiB of
+ * device memory, present on every GPU that loads the library until the process exits) for
+ * the partial output C[M,N], the tile flags, the task table and the status block.  Limits:
+ * M*N*2 bytes <= 8 MiB (for example 2048 x 2048) and control tables <= 1 MiB; a larger
+ * problem is rejected with ENTWINE_ERR_TOO_LARGE before anything is enqueued.
+ *
+ * Arguments as entwine_gemm_rs (all device pointers; `stream` a cudaStream_t), plus
+ *   status_out  NULL, or a host array of 8 values: the call then synchronises `stream` and
+ *               writes what entwine_last_status would (code, CTA, where, flags published,
+ *               tiles reduced, tiles pushed, T_G ns, T_end ns) and returns the code.
+ * The plan supplies the shape, order, budget and options; its own workspace is not touched
+ * and entwine_last_status does not report this call.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ * caches it per device: make that first call outside any stream capture.  All calls on a
+ * device share the one array, which keeps whatever the previous call left: every call first
+ * clears the flags, list heads and status on `stream`.  Two calls whose execution overlaps
+ * on the GPU (different streams, or different plans at once) therefore race; serialise them.
+ * Errors: ENTWINE_ERR_INVALID, ENTWINE_ERR_TOO_LARGE, ENTWINE_ERR_RESOURCES, ENTWINE_ERR_CUDA;
+ * with status_out also ENTWINE_ERR_TIMEOUT / ENTWINE_ERR_INTERNAL from the device.
+ */
+int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const void* B,
+                           const void* peer_partials, void* out_shard, void* send_bufs,
+                           void* stream, int64_t* status_out);
 
 /* entwine_destroy - free the plan and everything it owns (synchronises its last stream). */
 int entwine_destroy(entwine_plan_t plan);

@@ -1313,3 +1313,161 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, cons
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// entwine_gemm_rs_static: the fused call for callers that must not allocate
+// ------------------------------------------------------------------------------------------
+namespace entwine {
+
+// Scratch of the no-allocation entry point.  It lives in the library image: every device that
+// loads the library holds these 9 MiB until the process exits.  The first kStaticPartialMax
+// bytes hold the partial output C[M,N]; the rest holds the status block, the completion
+// counter, the list heads and offsets, the flag arrays and the task table.
+constexpr size_t kStaticPartialMax = size_t(8) << 20;
+constexpr size_t kStaticControlMax = size_t(1) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartialMax + kStaticControlMax];
+
+// Device address of g_static_scratch per device.  In host code the array's name is only a
+// stand-in for the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
+
+}  // namespace entwine
+
+extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const void* B,
+                                      const void* peer_partials, void* out_shard, void* send_bufs,
+                                      void* stream_v, int64_t* status_out) {
+  using namespace entwine;
+  if (!plan || !A || !B || !peer_partials || !out_shard || !send_bufs) return ENTWINE_ERR_INVALID;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(peer_partials) || !aligned16(out_shard) ||
+      !aligned16(send_bufs))
+    return ENTWINE_ERR_INVALID;
+  Plan* p = plan;
+  const Geometry& g = p->g;
+  const HostTables& t = p->tables;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+  // ---- sizes against the static maximum ----
+  const size_t c_bytes = size_t(g.M) * g.N * 2;
+  const size_t n_own = size_t(g.W) * g.Q, n_peer = size_t(g.W - 1) * g.Q;
+  const size_t off_status = 0;
+  const size_t off_done = off_status + align256(2 * sizeof(StatusSlot));
+  const size_t off_heads = off_done + 256;
+  const size_t off_offs = off_heads + align256(size_t(p->x) * 4);
+  const size_t off_fown = off_offs + align256(t.list_offs.size() * 4);
+  const size_t off_fpeer = off_fown + align256(n_own * 4);
+  const size_t off_tasks = off_fpeer + align256(n_peer * 4);
+  const size_t ctrl_bytes = off_tasks + align256(t.dev_tasks.size() * sizeof(Task));
+  if (c_bytes > kStaticPartialMax || ctrl_bytes > kStaticControlMax) return ENTWINE_ERR_TOO_LARGE;
+
+  // ---- once per device: the device address of the scratch symbol ----
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return ENTWINE_ERR_RESOURCES;
+  if (!g_static_scratch_addr[dev]) {
+    int major = 0, sms = 0;
+    CK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (major != 10) return ENTWINE_ERR_RESOURCES;
+    void* addr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&addr, g_static_scratch);
+    if (e != cudaSuccess || !addr) {
+      cudaGetLastError();
+      return ENTWINE_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
+  }
+  {
+    int sms = 0;
+    CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (p->num_sms > sms) return ENTWINE_ERR_RESOURCES;
+  }
+  unsigned char* base = g_static_scratch_addr[dev];
+  unsigned char* ctrl = base + kStaticPartialMax;
+
+  // ---- the array keeps the previous call's contents: reset what must start clean ----
+  static const StatusSlot kInit[2] = {{0, 0, 0, 0, ~0ULL, 0, 0, 0}, {0, 0, 0, 0, ~0ULL, 0, 0, 0}};
+  CK(cudaMemsetAsync(ctrl, 0, off_fpeer, stream));                      // status .. own flags
+  CK(cudaMemcpyAsync(ctrl + off_status, kInit, sizeof(kInit), cudaMemcpyHostToDevice, stream));
+  CK(cudaMemsetAsync(ctrl + off_fpeer, 0xff, n_peer * 4, stream));      // peers: pre-published
+  CK(cudaMemcpyAsync(ctrl + off_offs, t.list_offs.data(), t.list_offs.size() * 4, cudaMemcpyHostToDevice,
+                     stream));
+  CK(cudaMemcpyAsync(ctrl + off_tasks, t.dev_tasks.data(), t.dev_tasks.size() * sizeof(Task),
+                     cudaMemcpyHostToDevice, stream));
+  if (p->poison) CK(cudaMemsetAsync(base, 0xff, c_bytes, stream));
+
+  // ---- kernel arguments (same kernel as entwine_gemm_rs) ----
+  KParams kp;
+  std::memset(&kp, 0, sizeof(kp));
+  kp.M = int(g.M); kp.N = int(g.N); kp.K = int(g.K); kp.W = g.W; kp.r = p->rank; kp.order = p->order;
+  kp.rowsT = g.rowsT; kp.nBn = g.nBn; kp.nTn = g.nTn; kp.Lb = g.Lb; kp.P_blk = g.P_blk; kp.Q = g.Q;
+  kp.cpb = g.cpb; kp.R = g.R;
+  kp.x = p->x;
+  kp.mode = MODE_FUSED;
+  kp.help = p->tail_help;
+  kp.skip_wait = 0;
+  kp.epoch = 1;  // the flags were cleared above
+  kp.seq = 0;
+  kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
+  int rs = 64;
+  while (rs > 1 && int64_t(g.W) * rs * kTile * 2 > 32768) rs /= 2;
+  int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
+  int prs = rs;
+  while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
+  slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
+  if (slot_bytes * 2 > kRingBytes) return ENTWINE_ERR_RESOURCES;
+  kp.rs = rs;
+  kp.prs = prs;
+  kp.slot_bytes = slot_bytes;
+  kp.n_slots = std::min(kMaxSlots, kRingBytes / slot_bytes);
+  kp.status = reinterpret_cast<StatusSlot*>(ctrl + off_status);
+  kp.done_ctr = reinterpret_cast<unsigned*>(ctrl + off_done);
+  kp.list_head = reinterpret_cast<int*>(ctrl + off_heads);
+  kp.list_offs = reinterpret_cast<const int*>(ctrl + off_offs);
+  kp.flags_own = reinterpret_cast<unsigned*>(ctrl + off_fown);
+  kp.flags_peer = reinterpret_cast<const unsigned*>(ctrl + off_fpeer);
+  kp.tasks = reinterpret_cast<const Task*>(ctrl + off_tasks);
+  kp.G = p->n_gemm_ctas;
+  kp.n_ded = p->n_comm_ctas;
+  int grid = p->n_gemm_ctas + p->n_comm_ctas;
+  const bool pair = p->pair;
+  if (pair && (grid & 1)) {
+    if (grid + 1 > p->num_sms) grid -= 1, kp.n_ded -= 1;
+    else grid += 1, kp.n_ded += 1;
+    if (kp.n_ded < p->x) kp.help = 1;
+  }
+  KMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
+            make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
+            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.c_ld, base, g.M, g.N, kTile, rs, false) &&
+            make_map(&maps.p_ld, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, rs, false) &&
+            make_map(&maps.out_st, out_shard, g.R, g.N, kTile, rs, false) &&
+            make_map(&maps.send_st, send_bufs, int64_t(g.W - 1) * g.R, g.N, kTile, rs, false);
+  if (!ok) return ENTWINE_ERR_CUDA;
+  int rc;
+  if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
+  else if (g.BN == 256) rc = launch_bn<256, false>(p, kp, maps, grid, stream);
+  else rc = launch_bn<128, false>(p, kp, maps, grid, stream);
+  if (rc != ENTWINE_OK) return rc;
+
+  if (status_out) {
+    StatusSlot s;
+    CK(cudaStreamSynchronize(stream));
+    CK(cudaMemcpy(&s, ctrl + off_status, sizeof(s), cudaMemcpyDeviceToHost));
+    const int code = int(s.code_cta_task & 0xff);
+    status_out[0] = code ? -code : 0;
+    status_out[1] = int64_t((s.code_cta_task >> 8) & 0xffffff);
+    status_out[2] = int64_t(int32_t(s.code_cta_task >> 32));
+    status_out[3] = int64_t(s.flags_published);
+    status_out[4] = int64_t(s.tiles_reduced);
+    status_out[5] = int64_t(s.tiles_pushed);
+    status_out[6] = (s.t_gemm_end > s.t_start) ? int64_t(s.t_gemm_end - s.t_start) : 0;
+    status_out[7] = (s.t_end > s.t_start) ? int64_t(s.t_end - s.t_start) : 0;
+    return int(status_out[0]);
+  }
+  return ENTWINE_OK;
+}

@@ -299,6 +299,8 @@ const char* entwine_strerror(int code) {
     case ENTWINE_ERR_CUDA: return "CUDA call failed or no CUDA device";
     case ENTWINE_ERR_TIMEOUT: return "a device-side wait ran out of its budget";
     case ENTWINE_ERR_INTERNAL: return "a device-side index check failed";
+    case ENTWINE_ERR_TOO_LARGE:
+      return "problem exceeds the fixed scratch of entwine_gemm_rs_static (M*N*2 <= 8 MiB, tables <= 1 MiB)";
     default: return "unknown entwine error code";
   }
 }

@@ -22,6 +22,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 ORDER_ROW_MAJOR, ORDER_INTERLEAVED = 0, 1
 OK, ERR_INVALID, ERR_RESOURCES, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
+ERR_TOO_LARGE = -6
 OPT_RANK, OPT_BLOCK_N, OPT_WAIT_BUDGET_NS, OPT_TAIL_HELP = 1, 2, 3, 4
 OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL, OPT_PAIR_CTAS = 5, 6, 7, 8
 (EXPORT_COUNTS, EXPORT_ORDER, EXPORT_TILES, EXPORT_FLAG_SEQ, EXPORT_LIST_OFFS, EXPORT_TASKS,
@@ -30,7 +31,7 @@ OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL, OPT_PAIR_CTAS = 5, 6, 7, 8
 # every symbol include/entwine.h declares
 SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gemm_rs_host",
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
-           "entwine_last_status", "entwine_destroy", "entwine_strerror")
+           "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
@@ -43,6 +44,7 @@ _lib.entwine_read_partial.argtypes = [_vp, _vp, _vp]
 _lib.entwine_plan_export.argtypes = [_vp, _int, _vp, ctypes.POINTER(ctypes.c_size_t)]
 _lib.entwine_last_status.argtypes = [_vp, ctypes.POINTER(_i64)]
 _lib.entwine_destroy.argtypes = [_vp]
+_lib.entwine_gemm_rs_static.argtypes = [_vp] * 7 + [ctypes.POINTER(_i64)]
 _lib.entwine_strerror.argtypes = [_int]
 _lib.entwine_strerror.restype = ctypes.c_char_p
 for _name in SYMBOLS:
@@ -117,6 +119,21 @@ class Plan:
         """Host tensors (CPU, bf16, contiguous; pinned for speed)."""
         _check(_lib.entwine_gemm_rs_host(self._h, _ptr(A), _ptr(B), _ptr(peer_partials),
                                          _ptr(out_shard), _ptr(send_bufs)), "entwine_gemm_rs_host")
+
+    def gemm_rs_static(self, A, B, peer_partials, out_shard, send_bufs, stream=None, want_status=True):
+        """The fused call on the library's fixed scratch array: for callers that must not
+        allocate device memory (see include/entwine.h).  Problems above the array's limits raise
+        EntwineError(ERR_TOO_LARGE).  With want_status the call synchronises the stream and
+        returns the status dict; overlapping calls on one device race."""
+        out = (_i64 * 8)() if want_status else None
+        code = _lib.entwine_gemm_rs_static(self._h, _ptr(A), _ptr(B), _ptr(peer_partials), _ptr(out_shard),
+                                           _ptr(send_bufs), _stream(stream), out)
+        _check(code, "entwine_gemm_rs_static")
+        if not want_status:
+            return None
+        names = ("code", "cta", "where", "flags_published", "tiles_reduced", "tiles_pushed",
+                 "t_gemm_ns", "t_end_ns")
+        return {k: int(v) for k, v in zip(names, out)}
 
     def gemm_only(self, A, B, stream=None):
         _check(_lib.entwine_gemm_only(self._h, _ptr(A), _ptr(B), _stream(stream)), "entwine_gemm_only")
