@@ -248,6 +248,8 @@ def main():
     ap.add_argument("--impl", default="entwine", choices=["entwine", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--comm-ctas", type=int, default=0,
+                    help="with --kernel-only comm: number of consumer CTAs (0 = one per SM)")
     ap.add_argument("--kernel-only", default=None, choices=["fused", "gemm", "comm"],
                     help="profiling aid: run warmup+steps launches of one mode on the workload and exit")
     args = ap.parse_args()
@@ -286,7 +288,7 @@ def main():
         plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
         plan.gemm_only(A, Bm)
         fn = {"fused": lambda: plan.gemm_rs(A, Bm, P, out, send), "gemm": lambda: plan.gemm_only(A, Bm),
-              "comm": lambda: plan.comm_only(None, P, out, send, 0)}[args.kernel_only]
+              "comm": lambda: plan.comm_only(None, P, out, send, args.comm_ctas)}[args.kernel_only]
         us = time_steps(fn, args.steps, args.warmup, flush, torch)
         plan.last_status()
         print(json.dumps({"kernel_only": args.kernel_only, "workload": wl.name,

@@ -77,10 +77,15 @@ enum {
                                       there is no device)                                        */
   ENTWINE_OPT_POISON_PARTIAL  = 7, /* 1: fill the partial-output workspace with NaN patterns
                                       before each launch (ordering stress test; default 0)       */
-  ENTWINE_OPT_PAIR_CTAS       = 8  /* [pre] 1 (default): where the order allows it, two CTAs of a
+  ENTWINE_OPT_PAIR_CTAS       = 8, /* [pre] 1 (default): where the order allows it, two CTAs of a
                                       cluster compute a 256x256 pair tile (tcgen05 cta_group::2:
                                       two producer blocks that share a block column, each CTA
                                       loading half of the B panel); 0: every CTA works alone     */
+  ENTWINE_OPT_COLOCATE        = 9  /* 1 (default): with TAIL_HELP (or n_comm_sms = 0) a producer
+                                      CTA's consumer warps take tasks while its tensor-core work
+                                      is still running, through a small shared-memory ring beside
+                                      the producer's buffers (computation and communication share
+                                      the SM, Sec. 3.2); 0: they start when its last block is done */
 };
 
 /* What entwine_plan_export can write.  Integer tables, host memory, for bit-exact diffs. */

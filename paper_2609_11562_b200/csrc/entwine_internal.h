@@ -74,6 +74,7 @@ struct Plan {
   int num_sms = 148;
   bool num_sms_overridden = false;
   int tail_help = 1;
+  int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles
   bool pair = false;        // pair tiles in use for this plan
   int poison = 0;

@@ -15,21 +15,48 @@
 namespace entwine {
 
 // ------------------------------------------------------------------------------------------
-// compile-time shape of the producer
+// compile-time shape of the kernel
 // ------------------------------------------------------------------------------------------
 constexpr int kBM = 128;          // producer block rows = reduction tile rows
 constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes = one swizzle row)
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
-constexpr int kThreads = 320;     // producer: warp 0 TMA, warp 1 MMA + TMEM owner, warps 4-7 epilogue
-                                  // consumer: warp 0 polls flags + issues TMA loads, warps 1-8
-                                  // reduce, warp 9 issues the TMA stores
-constexpr int kEpiWarp0 = 4;
+// Warp roles of the 16 warps of a CTA.  Producer work (warps 0, 1, 4-7) and consumer work
+// (warps 2, 3, 8-15) run side by side in a producer CTA: the tensor pipe is driven by one
+// thread, so the SM's TMA and ALUs are free to move and reduce tiles meanwhile.
+constexpr int kThreads = 512;
+constexpr int kTmaWarp = 0;       // producer: TMA loads of A and B
+constexpr int kMmaWarp = 1;       // producer: tcgen05.mma issue, TMEM owner
+constexpr int kCommWarp = 2;      // consumer: claims tasks, polls flags, issues TMA loads
+constexpr int kStoreWarp = 3;     // consumer: TMA stores of pushed tiles, recycles ring slots
+constexpr int kEpiWarp0 = 4;      // producer: epilogue warps 4..7
 constexpr int kEpiThreads = 128;
-constexpr int kConsThreads = 256;
-constexpr int kStoreWarp = 9;
+constexpr int kRedWarp0 = 8;      // consumer: reducing warps 8..15
+constexpr int kRedThreads = 256;
+constexpr int kGemmThreads = 192; // warps 0, 1, 4-7
 constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abort flag
-constexpr int kMaxSlots = 8;          // consumer ring depth (upper bound)
 constexpr int kEpiStageBytes = 8192;  // per epilogue warp: 32 rows x 128 columns of bf16
+
+// Shared-memory map (offsets from a 1024-byte aligned base):
+//   [0, 163840)        operand ring of the producer (5 x 32 KiB, or 3 x 48 KiB)
+//   [163840, 196608)   epilogue staging (4 x 8 KiB)
+//   [196608, 229376)   consumer ring A: 2 slots of 16 KiB, used while the CTA still produces
+//   [0, 196608)        consumer ring B: 6 slots of 32 KiB, used once its producer work is over
+//   [229376, 230016)   mbarriers, TMEM base slot
+constexpr int kStageArea = 163840;
+constexpr int kStagingOff = kStageArea;
+constexpr int kRingAOff = kStagingOff + 4 * kEpiStageBytes;
+constexpr int kRingABytes = 32768;
+constexpr int kRingBOff = 0;
+constexpr int kRingBBytes = 196608;
+constexpr int kMaxSlots = 8;
+constexpr int kBarOff = kRingAOff + kRingABytes;
+constexpr int kBarBytes = 640;
+constexpr int kBarGemm = 0;        // full[<=6], empty[<=6], tfull[2], tempty[2]
+constexpr int kBarTmemSlot = 136;
+constexpr int kBarPair = 144;      // end-of-producer handshake of a CTA pair
+constexpr int kBarRingA = 192;     // full[8], empty[8], reduced[8]
+constexpr int kBarRingB = 192 + 192;
+constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
 
 // PAIR = two CTAs of a cluster compute a 256 x 256 pair tile with tcgen05 cta_group::2: each
 // CTA loads its own 128 rows of A and half (128 rows) of the B panel, so a CTA moves 32 KiB
@@ -41,22 +68,10 @@ struct Cfg {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = kBRows * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = 196608 / kStageBytes;  // 4 (128x256), 6 (128x128 or pair)
-  static constexpr int kPipeBytes = kStages * kStageBytes;
+  static constexpr int kStages = kStageArea / kStageBytes;  // 5 (pair, 128x128), 3 (128x256)
   static constexpr int kTmemCols = 2 * BN;  // two accumulators: epilogue overlaps next mainloop
+  static_assert(kStages >= 3 && kStages <= 6, "operand ring");
 };
-// Shared-memory map (offsets from a 1024-byte aligned base), identical for both block widths:
-//   [0, 196608)        producer: TMA/MMA operand ring          | consumer: tile ring
-//   [196608, 229376)   producer: epilogue staging (4 x 8 KiB)  | consumer: tile ring (cont.)
-//   [229376, 229888)   mbarriers + TMEM base slot
-constexpr int kPipeBytes = 196608;
-constexpr int kStagingOff = kPipeBytes;
-constexpr int kRingBytes = kPipeBytes + 4 * kEpiStageBytes;
-constexpr int kBarOff = kRingBytes;
-constexpr int kBarBytes = 512;
-constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
-static_assert(Cfg<256, false>::kPipeBytes == kPipeBytes && Cfg<128, false>::kPipeBytes == kPipeBytes &&
-                  Cfg<256, true>::kPipeBytes == kPipeBytes && Cfg<256, true>::kStages <= 8, "smem map");
 
 struct KParams {
   // geometry
@@ -68,16 +83,18 @@ struct KParams {
   int n_ded;      // CTAs [G, G + n_ded) are dedicated consumers
   int x;          // consumer lists
   int mode;       // Mode
-  int help;       // producers / finished consumers take tasks from other lists
+  int help;       // CTAs take tasks from lists other than their own
+  int colocate;   // a producer CTA's consumer warps work while it still produces
   int skip_wait;  // treat every flag as published (consumer in isolation)
-  int rs;         // rows of a tile moved per reduce step (all W contributions of those rows)
-  int prs;        // rows of a tile moved per push step
-  int slot_bytes; // bytes of one consumer ring slot
-  int n_slots;    // consumer ring depth
+  // consumer ring geometry, [0] ring A (small, beside the producer's buffers), [1] ring B
+  int rs[2];         // rows of a tile moved per reduce step (all W contributions of those rows)
+  int prs[2];        // rows of a tile moved per push step
+  int slot_bytes[2]; // bytes of one ring slot
   unsigned epoch;  // flag value of this producer run
   unsigned seq;    // launch counter: selects the status slot
   unsigned long long wait_budget_ns;
   // memory
+  __nv_bfloat16* out;            // out_shard [R][N] (written by the reducing warps)
   unsigned* flags_own;           // [W][Q]
   const unsigned* flags_peer;    // [W-1][Q]
   const Task* tasks;
@@ -92,10 +109,10 @@ struct KParams {
 struct KMaps {
   CUtensorMap a, b;      // operands
   CUtensorMap c_st;      // partial C, box 64 x 32, swizzled (epilogue stores)
-  CUtensorMap c_ld;      // partial C as the consumer reads it
-  CUtensorMap p_ld;      // incoming partials viewed as [(W-1)*M, N]
-  CUtensorMap out_st;    // out_shard [R, N]
-  CUtensorMap send_st;   // send_bufs viewed as [(W-1)*R, N]
+  // consumer maps, one set per ring (the box height is the ring's rs)
+  CUtensorMap c_ld[2];      // partial C as the consumer reads it
+  CUtensorMap p_ld[2];      // incoming partials viewed as [(W-1)*M, N]
+  CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N]
 };
 
 // ------------------------------------------------------------------------------------------
@@ -311,13 +328,14 @@ __device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) 
 // status helpers
 // ------------------------------------------------------------------------------------------
 struct SlotMeta {
-  int kind;      // 0 reduce step, 1 push tile, -1 end of work
+  int kind;      // 0 reduce step, 1 push step, -1 end of work, -2 continue on ring B
   int dst_x;     // column of the destination box
-  int dst_y;     // row of the destination box in the destination map
+  int dst_y;     // row of the destination box in the destination buffer
 };
 struct CtaShared {
-  volatile int abort;   // a role of this CTA (or another CTA) gave up
-  SlotMeta meta[kMaxSlots];
+  volatile int abort;      // a role of this CTA (or another CTA) gave up
+  volatile int gemm_done;  // this CTA's producer work is over; its shared memory is free
+  SlotMeta meta[2][kMaxSlots];
 };
 
 __device__ __forceinline__ void report(const KParams& P, int code, long long where) {
@@ -358,7 +376,7 @@ __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
       if (t0 == 0) t0 = now;
       else if (now - t0 > P.wait_budget_ns) return false;
     }
-    __nanosleep(32);
+    __nanosleep(64);
   }
 }
 
@@ -387,39 +405,79 @@ struct CommCounters {
   unsigned reduced = 0, pushed = 0;
 };
 
-// One CTA's consumer work: warp 0 claims tasks from `n_lists` consumer lists starting at
-// `first_list` (each list is consumed in order through its head counter, Sec. 3.1), polls
-// the tile flags with one lane per contributing rank, and streams the tiles through a ring
-// of shared-memory slots with TMA; warps 1-8 reduce the slots and warp 9 stores them.
-__device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
-                                  int first_list, int n_lists, CommCounters* cnt) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t ring_bar = smem_base + kBarOff + 256;
-  auto full_bar = [&](int s) { return ring_bar + 8u * s; };
-  auto empty_bar = [&](int s) { return ring_bar + 8u * (kMaxSlots + s); };
-  auto red_bar = [&](int s) { return ring_bar + 8u * (2 * kMaxSlots + s); };
-  const int rs = P.rs;
-  const int sub_bytes = rs * kTile * 2;      // one source's rows of one step
-  const int n_sub = kTile / rs;
+// A ring of shared-memory slots with its three barriers per slot.
+struct Ring {
+  uint32_t base;   // shared address of slot 0
+  uint32_t bars;   // shared address of full[kMaxSlots], empty[kMaxSlots], reduced[kMaxSlots]
+  int n_slots;
+  int id;          // 0 = ring A, 1 = ring B
+  int rs, prs, slot_bytes;
+  int sub_bytes;   // one contribution's rows of one reduce step
+  __device__ __forceinline__ uint32_t full(int s) const { return bars + 8u * s; }
+  __device__ __forceinline__ uint32_t empty(int s) const { return bars + 8u * (kMaxSlots + s); }
+  __device__ __forceinline__ uint32_t red(int s) const { return bars + 8u * (2 * kMaxSlots + s); }
+};
+__device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KParams& P) {
+  Ring r;
+  r.id = id;
+  r.base = smem_base + (id == 0 ? kRingAOff : kRingBOff);
+  r.bars = smem_base + kBarOff + (id == 0 ? kBarRingA : kBarRingB);
+  r.rs = P.rs[id];
+  r.prs = P.prs[id];
+  r.slot_bytes = P.slot_bytes[id];
+  r.sub_bytes = r.rs * kTile * 2;
+  r.n_slots = min(kMaxSlots, (id == 0 ? kRingABytes : kRingBBytes) / r.slot_bytes);
+  return r;
+}
 
-  if (warp == 0) {
+// One CTA's consumer work, run by warps 2, 3 and 8-15.  Warp 2 claims tasks from `n_lists`
+// consumer lists starting at `first_list` (each list is consumed in order through its head
+// counter, Sec. 3.1), polls the tile flags with one lane per contributing rank, and streams
+// the tiles through a ring of shared-memory slots with TMA; warps 8-15 reduce a slot in fp32
+// and write the result; warp 3 forwards pushed tiles with TMA stores and recycles the slots.
+// In a producer CTA the pipeline starts on the small ring A beside the producer's buffers and
+// moves to ring B (the producer's buffers) once `gemm_done` is set.
+__device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
+                                  int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P);
+
+  if (warp == kCommWarp) {
     // ---------------- claim, poll, load ----------------
     int it = 0;
     bool ok = true;
     const long long MN = (long long)P.M * P.N, RN = P.R * (long long)P.N;
+    // moves the pipeline to ring B once the producer's buffers are free
+    auto maybe_switch = [&]() {
+      if (ring.id != 0) return;
+      int done = 0;
+      if (lane == 0) done = sh->gemm_done;
+      done = __shfl_sync(0xffffffffu, done, 0);
+      if (!done) return;
+      bool free_slot = true;
+      if (lane == 0) {
+        const int slot = it % ring.n_slots;
+        free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+        if (free_slot) {
+          sh->meta[0][slot].kind = -2;
+          mbar_arrive(ring.full(slot));
+        }
+      }
+      ok = __all_sync(0xffffffffu, free_slot);
+      ring = make_ring(smem_base, 1, P);
+      it = 0;
+    };
     // Drains list j: claims go through the list's head counter, so the list is consumed in
-    // order whoever executes it.  The next claim is issued before the current task is
-    // processed, which hides the atomic's latency.
+    // order whoever executes it.  Two claims are kept in flight to hide the atomics' latency;
+    // a window of 32 task records (one per lane) is refilled when a claim falls outside it.
     auto drain = [&](int j) {
       const int base = P.list_offs[j];
       const int len = P.list_offs[j + 1] - base;
-      // two claims are kept in flight so that the atomics' latency is hidden
       int c0 = len, c1 = len;
       if (lane == 0) {
         c0 = atomicAdd(&P.list_head[j], 1);
         c1 = atomicAdd(&P.list_head[j], 1);
       }
-      // window of 32 task records, one per lane, refilled when a claim falls outside it
       int win = -(1 << 30);
       Task mine;
       mine.kind = 0; mine.d = 0; mine.t = 0; mine.slot = 0; mine.src_off = 0; mine.dst_off = 0;
@@ -465,55 +523,52 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
           }
           fence_async_all();  // the TMA reads below are ordered after the acquires
         }
+        maybe_switch();
+        if (!ok) break;
         const int trow = task.t / P.nTn, tcol = task.t % P.nTn;
         const int col = tcol * kTile;
         const int src_row = task.d * (int)P.R + trow * kTile;  // row of the tile in an [M,N] buffer
-        if (task.kind == 0) {
-          // one step = rs rows of all W contributions; lane q issues contribution q's load
-          for (int sub = 0; ok && sub < n_sub; ++sub, ++it) {
-            const int slot = it % P.n_slots;
-            const uint32_t ph = (it / P.n_slots) & 1;
-            bool free_slot = true;
-            if (lane == 0) {
-              free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
-              if (free_slot) {
-                sh->meta[slot].kind = 0;
-                sh->meta[slot].dst_x = col;
-                sh->meta[slot].dst_y = trow * kTile + sub * rs;
-                mbar_arrive_expect_tx(full_bar(slot), P.W * sub_bytes);
+        const int n_steps = kTile / (task.kind == 0 ? ring.rs : ring.prs);
+        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
+        for (int step = 0; ok && step < n_steps; ++step, ++it) {
+          const int slot = it % ring.n_slots;
+          const uint32_t ph = (it / ring.n_slots) & 1;
+          const uint32_t dst = ring.base + slot * ring.slot_bytes;
+          bool free_slot = true;
+          if (lane == 0) {
+            free_slot = mbar_wait(ring.empty(slot), ph ^ 1, P, sh);
+            if (free_slot) {
+              SlotMeta& m = sh->meta[ring.id][slot];
+              m.kind = task.kind;
+              m.dst_x = col;
+              if (task.kind == 0) {
+                m.dst_y = trow * kTile + step * rs;
+                mbar_arrive_expect_tx(ring.full(slot), P.W * sub_bytes);
+              } else {
+                m.dst_y = task.slot * (int)P.R + trow * kTile + step * ring.prs;
+                mbar_arrive_expect_tx(ring.full(slot), ring.prs * kTile * 2);
               }
             }
-            ok = __all_sync(0xffffffffu, free_slot);
-            if (!ok) break;
-            const uint32_t dst = smem_base + slot * P.slot_bytes;
-            // the local contribution first, then the peers in ascending rank order
+          }
+          ok = __all_sync(0xffffffffu, free_slot);
+          if (!ok) break;
+          if (task.kind == 0) {
+            // rs rows of the local contribution first, then of the peers in ascending rank
+            // order; lane q issues contribution q's load
             for (int q = lane; q < P.W; q += 32) {
-              if (q == 0) tma_load_2d(dst, &maps.c_ld, col, src_row + sub * rs, full_bar(slot));
-              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld, col, (q - 1) * P.M + src_row + sub * rs, full_bar(slot));
+              if (q == 0) tma_load_2d(dst, &maps.c_ld[ring.id], col, src_row + step * rs, ring.full(slot));
+              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld[ring.id], col, (q - 1) * P.M + src_row + step * rs,
+                               ring.full(slot));
             }
+          } else {
+            for (int rr = lane * rs; rr < ring.prs; rr += 32 * rs)
+              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld[ring.id], col, src_row + step * ring.prs + rr,
+                          ring.full(slot));
           }
-          if (lane == 0) cnt->reduced++;
-        } else {
-          for (int r0 = 0; ok && r0 < kTile; r0 += P.prs, ++it) {
-            const int slot = it % P.n_slots;
-            const uint32_t ph = (it / P.n_slots) & 1;
-            bool free_slot = true;
-            if (lane == 0) {
-              free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
-              if (free_slot) {
-                sh->meta[slot].kind = 1;
-                sh->meta[slot].dst_x = col;
-                sh->meta[slot].dst_y = task.slot * (int)P.R + trow * kTile + r0;
-                mbar_arrive_expect_tx(full_bar(slot), P.prs * kTile * 2);
-              }
-            }
-            ok = __all_sync(0xffffffffu, free_slot);
-            if (!ok) break;
-            const uint32_t dst = smem_base + slot * P.slot_bytes;
-            for (int rr = lane * rs; rr < P.prs; rr += 32 * rs)
-              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld, col, src_row + r0 + rr, full_bar(slot));
-          }
-          if (lane == 0) cnt->pushed++;
+        }
+        if (lane == 0) {
+          if (task.kind == 0) cnt->reduced++;
+          else cnt->pushed++;
         }
         if (!ok && lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
       }
@@ -541,80 +596,112 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       }
       if (!any) break;
     }
-    // end-of-work marker so that the reducing warps leave their loop
+    // end-of-work marker so that the other consumer warps leave their loops
     if (lane == 0) {
-      const int slot = it % P.n_slots;
-      const uint32_t ph = (it / P.n_slots) & 1;
-      const bool free_slot = mbar_wait(empty_bar(slot), ph ^ 1, P, sh);
+      const int slot = it % ring.n_slots;
+      const bool free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
       if (!free_slot) sh->abort = 1;
-      sh->meta[slot].kind = -1;
-      mbar_arrive(full_bar(slot));
+      sh->meta[ring.id][slot].kind = -1;
+      mbar_arrive(ring.full(slot));
     }
     __syncwarp();
-  } else if (warp <= kConsThreads / 32) {
+  } else if (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32) {
     // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
-    const int ctid = threadIdx.x - 32;
+    const int ctid = threadIdx.x - kRedWarp0 * 32;
     for (int it = 0;; ++it) {
-      const int slot = it % P.n_slots;
-      const uint32_t ph = (it / P.n_slots) & 1;
-      if (!mbar_wait(full_bar(slot), ph, P, sh)) {
+      const int slot = it % ring.n_slots;
+      const uint32_t ph = (it / ring.n_slots) & 1;
+      // one lane per warp polls; the warp-level vote carries the barrier's acquire to all lanes
+      bool landed = true;
+      if (lane == 0) landed = mbar_wait(ring.full(slot), ph, P, sh);
+      if (!__all_sync(0xffffffffu, landed)) {
         sh->abort = 1;
         break;
       }
-      const int kind = sh->meta[slot].kind;
-      if (kind < 0) break;
-      if (kind == 0) {
-        const uint32_t sbase = smem_base + slot * P.slot_bytes;
-        // start from the local contribution, add the peers in ascending rank order, fp32
-        for (int c = ctid; c < rs * (kTile * 2 / 16); c += kConsThreads) {
+      const SlotMeta m = sh->meta[ring.id][slot];
+      if (m.kind == -1) break;
+      if (m.kind == -2) {
+        ring = make_ring(smem_base, 1, P);
+        it = -1;
+        continue;
+      }
+      if (m.kind == 0) {
+        const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
+        __nv_bfloat16* dst = P.out + (long long)m.dst_y * P.N + m.dst_x;
+        // start from the local contribution, add the peers in ascending rank order, fp32; every
+        // thread writes its own 16 bytes of the output (single writer, 256-byte row segments)
+        for (int c = ctid; c < rs * (kTile * 2 / 16); c += kRedThreads) {
           float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
           const uint32_t addr = sbase + c * 16;
           acc_bf16x8(a, ld_shared_v4(addr));
 #pragma unroll 4
           for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
-          st_shared_v4(addr, pack_bf16x8(a));  // in place over the local contribution's rows
+          __stcs(reinterpret_cast<uint4*>(dst + (long long)(c >> 4) * P.N + (c & 15) * 8), pack_bf16x8(a));
         }
-        fence_async_smem();  // generic-proxy writes above -> visible to the TMA store
       }
-      // one arrival per warp hands the slot to the store warp (a push step is forwarded by the
-      // store warp alone; the arrival then only says that this warp has read the slot's header)
+      // one arrival per warp returns the slot (a push step is forwarded by the store warp alone;
+      // the arrival then only says that this warp has read the slot's header)
       __syncwarp();
-      if (lane == 0) mbar_arrive(red_bar(slot));
+      if (lane == 0) mbar_arrive(ring.red(slot));
     }
   } else if (warp == kStoreWarp && lane == 0) {
-    // ---------------- store the slots, recycle them ----------------
-    int prev_slot = -1;
+    // ---------------- forward push slots with TMA stores, recycle all slots ----------------
+    // Push stores are kept in flight: a pushed slot is released once its store has read it,
+    // which is awaited only when kPend younger stores exist or when this thread would idle.
+    constexpr int kPend = 3;
+    unsigned long long pend = 0;  // queue of barrier addresses' slot/ring ids, 8 bits each
+    int n_pend = 0;
+    auto retire_all = [&]() {
+      if (!n_pend) return;
+      bulk_wait_read<0>();
+      for (; n_pend > 0; --n_pend, pend >>= 8) {
+        const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P);
+        mbar_arrive(rr.empty(int(pend & 15u)));
+      }
+    };
     for (int it = 0;; ++it) {
-      const int slot = it % P.n_slots;
-      const uint32_t ph = (it / P.n_slots) & 1;
-      if (!mbar_wait(full_bar(slot), ph, P, sh)) {
+      const int slot = it % ring.n_slots;
+      const uint32_t ph = (it / ring.n_slots) & 1;
+      if (!mbar_try_wait(ring.full(slot), ph)) {
+        retire_all();  // nothing to do yet: let the stores in flight return their slots
+        if (!mbar_wait(ring.full(slot), ph, P, sh)) {
+          sh->abort = 1;
+          break;
+        }
+      }
+      const SlotMeta m = sh->meta[ring.id][slot];
+      if (m.kind == -1) break;
+      if (m.kind == -2) {
+        retire_all();
+        ring = make_ring(smem_base, 1, P);
+        it = -1;
+        continue;
+      }
+      const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+      if (!mbar_wait(ring.red(slot), ph, P, sh)) {
         sh->abort = 1;
         break;
       }
-      const int kind = sh->meta[slot].kind;
-      if (kind < 0) break;
-      const int dst_x = sh->meta[slot].dst_x, dst_y = sh->meta[slot].dst_y;
-      const uint32_t sbase = smem_base + slot * P.slot_bytes;
-      if (!mbar_wait(red_bar(slot), ph, P, sh)) {
-        sh->abort = 1;
-        break;
-      }
-      if (kind == 0) {
-        tma_store_2d(&maps.out_st, dst_x, dst_y, sbase);
+      if (m.kind == 0) {
+        mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
-        for (int rr = 0; rr < P.prs; rr += rs) tma_store_2d(&maps.send_st, dst_x, dst_y + rr, sbase + rr * kTile * 2);
+        for (int rr = 0; rr < ring.prs; rr += ring.rs)
+          tma_store_2d(&maps.send_st[ring.id], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2);
+        bulk_commit();
+        if (n_pend == kPend) {
+          bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
+          const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P);
+          mbar_arrive(rr.empty(int(pend & 15u)));
+          pend >>= 8;
+          --n_pend;
+        }
+        pend |= (unsigned long long)(unsigned(slot) | (unsigned(ring.id) << 4)) << (8 * n_pend);
+        ++n_pend;
       }
-      bulk_commit();
-      // the previous slot is free once its store has finished reading shared memory
-      if (prev_slot >= 0) {
-        bulk_wait_read<1>();
-        mbar_arrive(empty_bar(prev_slot));
-      }
-      prev_slot = slot;
     }
     bulk_wait_done<0>();  // every store of this CTA is complete before it exits
   }
-  __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -630,20 +717,27 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   StatusSlot* st = &P.status[P.seq & 1];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
-  const uint32_t bar_base = smem_base + kBarOff;
+  const uint32_t bar_base = smem_base + kBarOff + kBarGemm;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + 2 + a); };
-  const uint32_t tmem_slot = bar_base + 8u * (2 * C::kStages + 4);
+  const uint32_t tmem_slot = smem_base + kBarOff + kBarTmemSlot;
+  const uint32_t pair_bar = smem_base + kBarOff + kBarPair;
   const bool is_producer = (int)blockIdx.x < P.G && P.mode != MODE_COMM_ONLY;
   const int g = (int)blockIdx.x;                 // producer index
   const int cidx = (int)blockIdx.x - P.G;        // consumer index of a dedicated consumer CTA
   const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
   const bool leader = cta_rank == 0;
+  // work units of a producer: blocks p = g, g+G, ... or, for pairs, pair indices u = g/2, ...
+  const int n_units = PAIR ? P.P_blk / 2 : P.P_blk;
+  const int unit0 = PAIR ? g / 2 : g;
+  const int stride = PAIR ? P.G / 2 : P.G;
+  const int n_my = (is_producer && unit0 < n_units) ? (n_units - unit0 + stride - 1) / stride : 0;
 
   if (threadIdx.x == 0) {
     sh.abort = 0;
+    sh.gemm_done = (is_producer && n_my > 0) ? 0 : 1;
     atomicMin(&st->t_start, globaltimer_ns());
     if (is_producer) {
       for (int s = 0; s < C::kStages; ++s) {
@@ -654,34 +748,36 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         mbar_init(tfull_bar(a), 1);
         mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * (kEpiThreads / 32));
       }
+      mbar_init(pair_bar, 1);
     }
-    for (int s = 0; s < kMaxSlots; ++s) {  // consumer ring: full, empty, reduced
-      mbar_init(bar_base + 256 + 8u * s, 1);
-      mbar_init(bar_base + 256 + 8u * (kMaxSlots + s), 1);
-      mbar_init(bar_base + 256 + 8u * (2 * kMaxSlots + s), kConsThreads / 32);
+    for (int ring = 0; ring < 2; ++ring) {  // consumer rings: full, empty, reduced
+      const uint32_t rb = smem_base + kBarOff + (ring == 0 ? kBarRingA : kBarRingB);
+      for (int s = 0; s < kMaxSlots; ++s) {
+        mbar_init(rb + 8u * s, 1);
+        mbar_init(rb + 8u * (kMaxSlots + s), 1);
+        mbar_init(rb + 8u * (2 * kMaxSlots + s), kRedThreads / 32);
+      }
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (is_producer && warp == kMmaWarp) {
+    if (PAIR) tmem_alloc_pair(tmem_slot, C::kTmemCols);
+    else tmem_alloc(tmem_slot, C::kTmemCols);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (PAIR && is_producer) cluster_sync_all();  // both CTAs' barriers exist before either signals
+  tc_fence_after();
+
   CommCounters cnt;
   unsigned published = 0;
+  const bool gemm_warp = warp == kTmaWarp || warp == kMmaWarp || (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4);
+  const bool comm_warp = warp == kCommWarp || warp == kStoreWarp || warp >= kRedWarp0;
 
-  if (is_producer) {
+  if (is_producer && gemm_warp) {
     // ---------------- producer: tcgen05 GEMM ----------------
-    if (warp == 1) {
-      if (PAIR) tmem_alloc_pair(tmem_slot, C::kTmemCols);
-      else tmem_alloc(tmem_slot, C::kTmemCols);
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other
-    tc_fence_after();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + kBarOff + 8 * (2 * C::kStages + 4));
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + kBarOff + kBarTmemSlot);
     const int KB = (P.K + kBK - 1) / kBK;
-    // work units: blocks p = g, g+G, ... or, for pairs, pair indices u = g/2, g/2 + G/2, ...
-    const int n_units = PAIR ? P.P_blk / 2 : P.P_blk;
-    const int unit0 = PAIR ? g / 2 : g;
-    const int stride = PAIR ? P.G / 2 : P.G;
-    const int n_my = (unit0 < n_units) ? (n_units - unit0 + stride - 1) / stride : 0;
     auto block_of = [&](int i, int* d, int* l) {
       const int unit = unit0 + i * stride;
       const int p = PAIR ? pair_position(P, unit, (int)cta_rank) : unit;
@@ -689,7 +785,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       else { *d = p / P.Lb; *l = p - *d * P.Lb; }
     };
 
-    if (warp == 0 && lane == 0) {
+    if (warp == kTmaWarp && lane == 0) {
       // ---- TMA producer (every CTA loads its own operands) ----
       int stage = 0;
       uint32_t phase = 0;
@@ -716,7 +812,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         }
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -1); }
-    } else if (warp == 1 && lane == 0 && leader) {
+    } else if (warp == kMmaWarp && lane == 0 && leader) {
       // ---- MMA issuer (the leader CTA issues for the pair) ----
       int stage = 0;
       uint32_t phase = 0;
@@ -751,7 +847,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -2); }
-    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiThreads / 32) {
+    } else if (warp >= kEpiWarp0) {
       // ---- epilogue: TMEM -> bf16 -> swizzled staging -> TMA store of the partial C, then the
       //      block's tile flags ----
       const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
@@ -826,51 +922,71 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       }
       if (!ok && lane == 0) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -3); }
     }
-    __syncthreads();
-    if (threadIdx.x == 0 && n_my > 0) atomicMax(&st->t_gemm_end, globaltimer_ns());
+    // ---- end of this CTA's producer work ----
+    named_bar_sync(3, kGemmThreads);
+    if (warp == kTmaWarp && lane == 0 && n_my > 0) atomicMax(&st->t_gemm_end, globaltimer_ns());
     if (sh.abort) {
       // give copies that may still be in flight time to land before the CTA's memory is reused
       const unsigned long long t0 = globaltimer_ns();
       while (globaltimer_ns() - t0 < 200000ULL) __nanosleep(1000);
     }
-    // the peer may still read this CTA's operands / signal its barriers until it is done too
-    if (PAIR) cluster_sync_all();
+    if (PAIR) {
+      // the peer may still signal this CTA's barriers until its producer warps are done too
+      if (warp == kMmaWarp && lane == 0) {
+        mbar_arrive_cluster(map_to_cta(pair_bar, cta_rank ^ 1));
+        if (!mbar_wait(pair_bar, 0, P, &sh)) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -4); }
+      }
+      named_bar_sync(3, kGemmThreads);
+    }
     tc_fence_after();
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
       if (PAIR) tmem_dealloc_pair(tmem_base, C::kTmemCols);
       else tmem_dealloc(tmem_base, C::kTmemCols);
     }
-    __syncthreads();
-  } else {
-    __syncthreads();  // barrier initialisation visible to the whole CTA
-  }
-
-  // ---------------- consumer ----------------
-  if (P.mode != MODE_GEMM_ONLY && !sh.abort) {
+    if (warp == kTmaWarp && lane == 0) {
+      __threadfence_block();
+      sh.gemm_done = 1;  // the consumer warps may take over the producer's shared memory
+    }
+    if (warp == kEpiWarp0 && lane == 0 && published)
+      atomicAdd(&st->flags_published, (unsigned long long)published);
+  } else if (comm_warp && P.mode != MODE_GEMM_ONLY) {
+    // ---------------- consumer ----------------
     int first = 0, count = 0;
+    bool on_a = false;
     if (!is_producer) {
       // dedicated consumer block j: its own list, then (shared-pool analogue) the others
       first = cidx % P.x;
       count = (cidx < P.x && !P.help) ? 1 : P.x;
-    } else if (P.n_ded == 0) {
-      // non-overlapped use of all SMs: block g consumes list g (then helps)
-      first = g % P.x;
-      count = P.help ? P.x : (g < P.x ? 1 : 0);
-    } else if (P.help) {
-      first = g % P.x;
-      count = P.x;
+    } else {
+      if (P.n_ded == 0) {
+        // no dedicated consumers: block g owns list g (and helps with the others)
+        first = g % P.x;
+        count = P.help ? P.x : (g < P.x ? 1 : 0);
+      } else if (P.help) {
+        first = g % P.x;
+        count = P.x;
+      }
+      on_a = n_my > 0;
+      if (count > 0 && on_a && !P.colocate) {
+        // not co-located: wait for the CTA's producer work to end, then use ring B
+        unsigned long long t0 = globaltimer_ns();
+        while (!sh.gemm_done && !sh.abort) {
+          __nanosleep(256);
+          if (globaltimer_ns() - t0 > 64ULL * P.wait_budget_ns) break;
+        }
+        on_a = false;
+      }
     }
-    if (count > 0) consumer_pipeline(P, maps, &sh, smem_base, first, count, &cnt);
+    if (count > 0 && !sh.abort) consumer_pipeline(P, maps, &sh, smem_base, first, count, on_a, &cnt);
+    if (warp == kCommWarp && lane == 0) {
+      if (cnt.reduced) atomicAdd(&st->tiles_reduced, (unsigned long long)cnt.reduced);
+      if (cnt.pushed) atomicAdd(&st->tiles_pushed, (unsigned long long)cnt.pushed);
+    }
   }
 
   // ---------------- exit bookkeeping ----------------
   __syncthreads();
-  if (is_producer && warp == kEpiWarp0 && lane == 0 && published)
-    atomicAdd(&st->flags_published, (unsigned long long)published);
-  __syncthreads();
   if (threadIdx.x == 0) {
-    if (cnt.reduced) atomicAdd(&st->tiles_reduced, (unsigned long long)cnt.reduced);
-    if (cnt.pushed) atomicAdd(&st->tiles_pushed, (unsigned long long)cnt.pushed);
     atomicMax(&st->t_end, globaltimer_ns());
     __threadfence();
     const unsigned prev = atomicAdd(P.done_ctr, 1u);
@@ -1081,6 +1197,23 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   return ENTWINE_OK;
 }
 
+// Consumer ring geometry: a reduce step moves rs rows of all W contributions (at most 16 KiB
+// on ring A, 32 KiB on ring B), a push step moves as many rows of one tile as fit in a slot.
+static void ring_geometry(const Geometry& g, KParams* kp) {
+  for (int id = 0; id < 2; ++id) {
+    const int budget = id == 0 ? 16384 : 32768;
+    int rs = 1;
+    while (int64_t(g.W) * (rs * 2) * kTile * 2 <= budget && rs * 2 <= kTile) rs *= 2;
+    int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
+    slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
+    int prs = rs;
+    while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
+    kp->rs[id] = rs;
+    kp->prs[id] = prs;
+    kp->slot_bytes[id] = slot_bytes;
+  }
+}
+
 // Common launch path.  `partial` overrides the workspace in consumer-only mode.
 static int launch(Plan* p, int mode, const void* A, const void* B, const void* partial, const void* peers,
                   void* out, void* send, int n_ctas, cudaStream_t stream) {
@@ -1133,19 +1266,9 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   d->seq += 1;
   kp.seq = d->seq;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  // consumer ring: a reduce step moves rs rows of all W contributions (about 32 KiB), a push
-  // step moves as many rows of one tile as fit in the same slot
-  int rs = 64;
-  while (rs > 1 && int64_t(g.W) * rs * kTile * 2 > 32768) rs /= 2;
-  int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
-  int prs = rs;
-  while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
-  slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
-  if (slot_bytes * 2 > kRingBytes) return ENTWINE_ERR_RESOURCES;
-  kp.rs = rs;
-  kp.prs = prs;
-  kp.slot_bytes = slot_bytes;
-  kp.n_slots = std::min(kMaxSlots, kRingBytes / slot_bytes);
+  ring_geometry(g, &kp);
+  kp.colocate = p->colocate;
+  kp.out = static_cast<__nv_bfloat16*>(out);
   kp.flags_own = d->flags_own;
   kp.flags_peer = d->flags_peer;
   kp.tasks = d->tasks;
@@ -1191,11 +1314,13 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
                      kBK, kBM, true) &&
             make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
                      kBK, (mode != MODE_COMM_ONLY) ? (pair ? 128 : g.BN) : kBM, true) &&
-            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true) &&
-            make_map(&maps.c_ld, c_src, g.M, g.N, kTile, rs, false) &&
-            make_map(&maps.p_ld, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, rs, false) &&
-            make_map(&maps.out_st, comm ? out : d->C, comm ? g.R : g.M, g.N, kTile, rs, false) &&
-            make_map(&maps.send_st, comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, rs, false);
+            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true);
+  for (int id = 0; ok && id < 2; ++id) {
+    const int rs = kp.rs[id];
+    ok = make_map(&maps.c_ld[id], c_src, g.M, g.N, kTile, rs, false) &&
+         make_map(&maps.p_ld[id], comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, rs, false) &&
+         make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, rs, false);
+  }
   if (!ok) return ENTWINE_ERR_CUDA;
   if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
   else if (g.BN == 256) rc = launch_bn<256, false>(p, kp, maps, grid, stream);
@@ -1411,17 +1536,9 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  int rs = 64;
-  while (rs > 1 && int64_t(g.W) * rs * kTile * 2 > 32768) rs /= 2;
-  int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
-  int prs = rs;
-  while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
-  slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
-  if (slot_bytes * 2 > kRingBytes) return ENTWINE_ERR_RESOURCES;
-  kp.rs = rs;
-  kp.prs = prs;
-  kp.slot_bytes = slot_bytes;
-  kp.n_slots = std::min(kMaxSlots, kRingBytes / slot_bytes);
+  ring_geometry(g, &kp);
+  kp.colocate = p->colocate;
+  kp.out = static_cast<__nv_bfloat16*>(out_shard);
   kp.status = reinterpret_cast<StatusSlot*>(ctrl + off_status);
   kp.done_ctr = reinterpret_cast<unsigned*>(ctrl + off_done);
   kp.list_head = reinterpret_cast<int*>(ctrl + off_heads);
@@ -1442,11 +1559,13 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   std::memset(&maps, 0, sizeof(maps));
   bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
             make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
-            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true) &&
-            make_map(&maps.c_ld, base, g.M, g.N, kTile, rs, false) &&
-            make_map(&maps.p_ld, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, rs, false) &&
-            make_map(&maps.out_st, out_shard, g.R, g.N, kTile, rs, false) &&
-            make_map(&maps.send_st, send_bufs, int64_t(g.W - 1) * g.R, g.N, kTile, rs, false);
+            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true);
+  for (int id = 0; ok && id < 2; ++id) {
+    const int rs = kp.rs[id];
+    ok = make_map(&maps.c_ld[id], base, g.M, g.N, kTile, rs, false) &&
+         make_map(&maps.p_ld[id], peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, rs, false) &&
+         make_map(&maps.send_st[id], send_bufs, int64_t(g.W - 1) * g.R, g.N, kTile, rs, false);
+  }
   if (!ok) return ENTWINE_ERR_CUDA;
   int rc;
   if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);

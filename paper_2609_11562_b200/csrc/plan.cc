@@ -248,6 +248,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       }
       return rc;
     }
+    case ENTWINE_OPT_COLOCATE:
+      if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
+      p->colocate = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_PAIR_CTAS:
       if (p->launched || (value != 0 && value != 1)) return ENTWINE_ERR_INVALID;
       p->pair_opt = int(value);
