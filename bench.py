@@ -239,6 +239,49 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     return res
 
 
+def run_sweep(args, peaks, flush, torch, E, I):
+    """The sweep configuration: every shape x communication budget x tile order, fused call only.
+    One JSON line per point goes to --sweep-out; stdout gets one summary line."""
+    os.makedirs(os.path.dirname(args.sweep_out), exist_ok=True)
+    n_points, best = 0, {}
+    with open(args.sweep_out, "w") as f:
+        for wl in I.sweep_workloads():
+            A, Bm = I.make_operands(wl, device="cuda")
+            P = I.make_peer_partials(wl, device="cuda")
+            out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+            send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+            tc, hb = roofline_seconds(wl, peaks)
+            for order in (1, 0):
+                for n_comm in I.SWEEP_COMM_SMS:
+                    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=wl.W - 1)
+                    us = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), args.sweep_iters, 2, flush, torch)
+                    st = plan.last_status()
+                    c = plan.counts()
+                    assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+                    med = statistics.median(us)
+                    rec = {"M": wl.M, "N": wl.N, "K_local": wl.K, "W": wl.W, "n_comm_sms": n_comm,
+                           "tile_order": "interleaved" if order else "row_major", "fused_us": med,
+                           "tflops": wl.flops / med / 1e6, "roofline_us": max(tc, hb) * 1e6,
+                           "roofline_frac": max(tc, hb) * 1e6 / med, "bound": "tensor" if tc >= hb else "hbm",
+                           "t_gemm_us": st["t_gemm_ns"] / 1e3, "t_end_us": st["t_end_ns"] / 1e3}
+                    f.write(json.dumps(rec) + "\n")
+                    n_points += 1
+                    key = (wl.M, wl.K, wl.W)
+                    if key not in best or med < best[key]["fused_us"]:
+                        best[key] = rec
+                    plan.destroy()
+            del A, Bm, P, out, send
+            torch.cuda.empty_cache()
+    fr = [b["roofline_frac"] for b in best.values()]
+    inter = sum(1 for b in best.values() if b["tile_order"] == "interleaved")
+    print(json.dumps({"sweep_points": n_points, "shapes": len(best), "out": args.sweep_out,
+                      "best_roofline_frac": {"min": min(fr), "median": statistics.median(fr), "max": max(fr)},
+                      "shapes_where_interleaved_is_best": inter,
+                      "best_budget_histogram": {str(k): sum(1 for b in best.values() if b["n_comm_sms"] == k)
+                                                for k in I.SWEEP_COMM_SMS}}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -248,6 +291,11 @@ def main():
     ap.add_argument("--impl", default="entwine", choices=["entwine", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="run the sweep configuration (60 shapes x budgets 0..32 x both orders), write one "
+                         "JSON line per point to --sweep-out and print a summary line")
+    ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
+    ap.add_argument("--sweep-iters", type=int, default=8)
     ap.add_argument("--comm-ctas", type=int, default=0,
                     help="with --kernel-only comm: number of consumer CTAs (0 = one per SM)")
     ap.add_argument("--kernel-only", default=None, choices=["fused", "gemm", "comm"],
@@ -280,6 +328,8 @@ def main():
 
     peaks = load_peaks()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB of L2
+    if args.sweep:
+        return run_sweep(args, peaks, flush, torch, E, I)
     if args.kernel_only:
         A, Bm = I.make_operands(wl, device="cuda")
         P = I.make_peer_partials(wl, device="cuda")

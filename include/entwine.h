@@ -81,6 +81,11 @@ enum {
                                       cluster compute a 256x256 pair tile (tcgen05 cta_group::2:
                                       two producer blocks that share a block column, each CTA
                                       loading half of the B panel); 0: every CTA works alone     */
+  ENTWINE_OPT_PREFETCH        = 10, /* 1: the consumer's polling warp prefetches the next reduce
+                                      task's published peer tiles into L2; 0 (default): off      */
+  ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
+                                      memory they leave goes to the co-located consumer ring;
+                                      0 (default): chosen from the shape                         */
   ENTWINE_OPT_COLOCATE        = 9  /* 1 (default): with TAIL_HELP (or n_comm_sms = 0) a producer
                                       CTA's consumer warps take tasks while its tensor-core work
                                       is still running, through a small shared-memory ring beside

@@ -74,6 +74,8 @@ struct Plan {
   int num_sms = 148;
   bool num_sms_overridden = false;
   int tail_help = 1;
+  int prefetch = 0;         // look-ahead L2 prefetch of peer tiles (measured: no gain)
+  int stages = 0;           // operand-ring stages of the producer, 0 = choose
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles
   bool pair = false;        // pair tiles in use for this plan

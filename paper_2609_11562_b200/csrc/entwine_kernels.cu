@@ -36,22 +36,24 @@ constexpr int kGemmThreads = 192; // warps 0, 1, 4-7
 constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abort flag
 constexpr int kEpiStageBytes = 8192;  // per epilogue warp: 32 rows x 128 columns of bf16
 
-// Shared-memory map (offsets from a 1024-byte aligned base):
-//   [0, 163840)        operand ring of the producer (5 x 32 KiB, or 3 x 48 KiB)
-//   [163840, 196608)   epilogue staging (4 x 8 KiB)
-//   [196608, 229376)   consumer ring A: 2 slots of 16 KiB, used while the CTA still produces
-//   [0, 196608)        consumer ring B: 6 slots of 32 KiB, used once its producer work is over
-//   [229376, 230016)   mbarriers, TMEM base slot
-constexpr int kStageArea = 163840;
-constexpr int kStagingOff = kStageArea;
-constexpr int kRingAOff = kStagingOff + 4 * kEpiStageBytes;
-constexpr int kRingABytes = 32768;
+// Shared-memory map (offsets from a 1024-byte aligned base).  The first 224 KiB are split at
+// launch time between the producer's operand ring (S stages), the epilogue staging and the
+// consumer's ring A, which a producer CTA's consumer warps use while it still produces:
+//   [0, S*stage)                operand ring of the producer
+//   [S*stage, S*stage + 32 KiB) epilogue staging (4 x 8 KiB)
+//   [.., 229376)                consumer ring A (32 KiB with 5 pair stages, 64 KiB with 4, ...)
+//   [0, 196608)                 consumer ring B: 6 slots of 32 KiB, used once the CTA's producer
+//                               work is over (and by dedicated consumer CTAs from the start)
+//   [229376, 230016)            mbarriers, TMEM base slot
+constexpr int kDataBytes = 229376;
+constexpr int kStagingBytes = 4 * kEpiStageBytes;
 constexpr int kRingBOff = 0;
 constexpr int kRingBBytes = 196608;
 constexpr int kMaxSlots = 8;
-constexpr int kBarOff = kRingAOff + kRingABytes;
+constexpr int kMaxStages = 6;
+constexpr int kBarOff = kDataBytes;
 constexpr int kBarBytes = 640;
-constexpr int kBarGemm = 0;        // full[<=6], empty[<=6], tfull[2], tempty[2]
+constexpr int kBarGemm = 0;        // full[6], empty[6], tfull[2], tempty[2]
 constexpr int kBarTmemSlot = 136;
 constexpr int kBarPair = 144;      // end-of-producer handshake of a CTA pair
 constexpr int kBarRingA = 192;     // full[8], empty[8], reduced[8]
@@ -68,9 +70,7 @@ struct Cfg {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = kBRows * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = kStageArea / kStageBytes;  // 5 (pair, 128x128), 3 (128x256)
   static constexpr int kTmemCols = 2 * BN;  // two accumulators: epilogue overlaps next mainloop
-  static_assert(kStages >= 3 && kStages <= 6, "operand ring");
 };
 
 struct KParams {
@@ -85,6 +85,10 @@ struct KParams {
   int mode;       // Mode
   int help;       // CTAs take tasks from lists other than their own
   int colocate;   // a producer CTA's consumer warps work while it still produces
+  int prefetch;   // pull the next reduce task's peer tiles into L2 ahead of its loads
+  int stages;     // operand-ring stages of the producer
+  int ring_a_off, ring_a_bytes;  // consumer ring A (after the epilogue staging)
+  int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
   int skip_wait;  // treat every flag as published (consumer in isolation)
   // consumer ring geometry, [0] ring A (small, beside the producer's buffers), [1] ring B
   int rs[2];         // rows of a tile moved per reduce step (all W contributions of those rows)
@@ -113,6 +117,7 @@ struct KMaps {
   CUtensorMap c_ld[2];      // partial C as the consumer reads it
   CUtensorMap p_ld[2];      // incoming partials viewed as [(W-1)*M, N]
   CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N]
+  CUtensorMap p_pf;         // incoming partials, whole-tile box, for L2 prefetch
 };
 
 // ------------------------------------------------------------------------------------------
@@ -158,6 +163,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
@@ -411,6 +420,7 @@ struct Ring {
   uint32_t bars;   // shared address of full[kMaxSlots], empty[kMaxSlots], reduced[kMaxSlots]
   int n_slots;
   int id;          // 0 = ring A, 1 = ring B
+  int geom;        // index of the step geometry and of the tensor-map set
   int rs, prs, slot_bytes;
   int sub_bytes;   // one contribution's rows of one reduce step
   __device__ __forceinline__ uint32_t full(int s) const { return bars + 8u * s; }
@@ -420,13 +430,14 @@ struct Ring {
 __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KParams& P) {
   Ring r;
   r.id = id;
-  r.base = smem_base + (id == 0 ? kRingAOff : kRingBOff);
+  r.geom = id == 0 ? P.ring_a_geom : 1;
+  r.base = smem_base + (id == 0 ? P.ring_a_off : kRingBOff);
   r.bars = smem_base + kBarOff + (id == 0 ? kBarRingA : kBarRingB);
-  r.rs = P.rs[id];
-  r.prs = P.prs[id];
-  r.slot_bytes = P.slot_bytes[id];
+  r.rs = P.rs[r.geom];
+  r.prs = P.prs[r.geom];
+  r.slot_bytes = P.slot_bytes[r.geom];
   r.sub_bytes = r.rs * kTile * 2;
-  r.n_slots = min(kMaxSlots, (id == 0 ? kRingABytes : kRingBBytes) / r.slot_bytes);
+  r.n_slots = min(kMaxSlots, (id == 0 ? P.ring_a_bytes : kRingBBytes) / r.slot_bytes);
   return r;
 }
 
@@ -507,6 +518,25 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
           if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
           continue;
         }
+        if (P.prefetch) {
+          // Look-ahead: the claim after this one names the next task.  If it is a reduce task
+          // whose peer contributions are already published, pull their tiles into L2 now (one
+          // lane per peer) so that the ring's loads find them there while holding a slot.
+          const int nx = __shfl_sync(0xffffffffu, c0, 0);
+          if (nx < len && nx >= win && nx < win + 32) {
+            const int lk = nx - win;
+            const int nkind = __shfl_sync(0xffffffffu, mine.kind, lk);
+            const int nd = __shfl_sync(0xffffffffu, mine.d, lk);
+            const int nt = __shfl_sync(0xffffffffu, mine.t, lk);
+            if (nkind == 0 && nt >= 0 && nt < P.Q && nd >= 0 && nd < P.W) {
+              const int nrow = nd * (int)P.R + (nt / P.nTn) * kTile, ncol = (nt % P.nTn) * kTile;
+              for (int q = lane - 1; q >= 0 && q < P.W - 1; q += 31) {
+                if (P.skip_wait || ld_acquire_gpu(&P.flags_peer[q * P.Q + nt]) >= P.epoch)
+                  tma_prefetch_l2_2d(&maps.p_pf, ncol, q * P.M + nrow);
+              }
+            }
+          }
+        }
         if (!P.skip_wait) {
           // lane 0 polls the local flag, lanes 1.. the peers' flags in rank order (Sec. 4.2);
           // the warp proceeds when all W contributions of the tile are published
@@ -556,13 +586,13 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
             // rs rows of the local contribution first, then of the peers in ascending rank
             // order; lane q issues contribution q's load
             for (int q = lane; q < P.W; q += 32) {
-              if (q == 0) tma_load_2d(dst, &maps.c_ld[ring.id], col, src_row + step * rs, ring.full(slot));
-              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld[ring.id], col, (q - 1) * P.M + src_row + step * rs,
+              if (q == 0) tma_load_2d(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot));
+              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld[ring.geom], col, (q - 1) * P.M + src_row + step * rs,
                                ring.full(slot));
             }
           } else {
             for (int rr = lane * rs; rr < ring.prs; rr += 32 * rs)
-              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld[ring.id], col, src_row + step * ring.prs + rr,
+              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld[ring.geom], col, src_row + step * ring.prs + rr,
                           ring.full(slot));
           }
         }
@@ -687,7 +717,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
         for (int rr = 0; rr < ring.prs; rr += ring.rs)
-          tma_store_2d(&maps.send_st[ring.id], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2);
+          tma_store_2d(&maps.send_st[ring.geom], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2);
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
@@ -719,9 +749,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_base + kBarOff + kBarGemm;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + 2 + a); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + 2 + a); };
+  const int n_stages = P.stages;
   const uint32_t tmem_slot = smem_base + kBarOff + kBarTmemSlot;
   const uint32_t pair_bar = smem_base + kBarOff + kBarPair;
   const bool is_producer = (int)blockIdx.x < P.G && P.mode != MODE_COMM_ONLY;
@@ -740,7 +771,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     sh.gemm_done = (is_producer && n_my > 0) ? 0 : 1;
     atomicMin(&st->t_start, globaltimer_ns());
     if (is_producer) {
-      for (int s = 0; s < C::kStages; ++s) {
+      for (int s = 0; s < n_stages; ++s) {
         mbar_init(full_bar(s), 1);
         mbar_init(empty_bar(s), 1);
       }
@@ -808,7 +839,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
             tma_load_2d(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage));
             tma_load_2d(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage));
           }
-          if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -1); }
@@ -839,7 +870,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (PAIR) tc_commit_pair(empty_bar(stage));
           else tc_commit(empty_bar(stage));
-          if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+          if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
         if (PAIR) tc_commit_pair(tfull_bar(acc));  // accumulator complete (both CTAs' halves)
@@ -851,7 +882,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       // ---- epilogue: TMEM -> bf16 -> swizzled staging -> TMA store of the partial C, then the
       //      block's tile flags ----
       const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
-      const uint32_t stg = smem_base + kStagingOff + q * kEpiStageBytes;
+      const uint32_t stg = smem_base + n_stages * C::kStageBytes + q * kEpiStageBytes;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
@@ -1197,9 +1228,12 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   return ENTWINE_OK;
 }
 
-// Consumer ring geometry: a reduce step moves rs rows of all W contributions (at most 16 KiB
-// on ring A, 32 KiB on ring B), a push step moves as many rows of one tile as fit in a slot.
-static void ring_geometry(const Geometry& g, KParams* kp) {
+// Consumer ring geometry and the split of shared memory.  A reduce step moves rs rows of all W
+// contributions (at most 16 KiB with geometry 0, 32 KiB with geometry 1), a push step moves as
+// many rows of one tile as fit in a slot.  The producer's operand ring gets `stages` stages;
+// what remains after the epilogue staging is the co-located consumer ring A.
+static int ring_geometry(const Plan* p, KParams* kp) {
+  const Geometry& g = p->g;
   for (int id = 0; id < 2; ++id) {
     const int budget = id == 0 ? 16384 : 32768;
     int rs = 1;
@@ -1212,6 +1246,26 @@ static void ring_geometry(const Geometry& g, KParams* kp) {
     kp->prs[id] = prs;
     kp->slot_bytes[id] = slot_bytes;
   }
+  const int stage_bytes = kBM * kBK * 2 + (p->pair ? 128 : g.BN) * kBK * 2;
+  int stages = p->stages;
+  if (stages <= 0) {
+    // default: deep operand ring; shapes whose communication outweighs their tensor work give
+    // one stage to the co-located consumer ring
+    stages = (kDataBytes - kStagingBytes - 2 * kp->slot_bytes[0]) / stage_bytes;
+    if (stages > 5) stages = 5;
+    const double t_tc = 2.0 * g.M * g.N * g.K / 1.6e15;
+    const double t_hbm = double(g.M) * g.N * 2.0 * (3 * g.W - 1) / g.W / 6.5e12;
+    if (p->colocate && t_hbm > 0.5 * t_tc && stages > 3) stages -= 1;
+  }
+  if (stages < 2 || stages > kMaxStages) return ENTWINE_ERR_INVALID;
+  const int ring_a_off = stages * stage_bytes + kStagingBytes;
+  const int ring_a_bytes = kDataBytes - ring_a_off;
+  if (ring_a_bytes < 2 * kp->slot_bytes[0]) return ENTWINE_ERR_RESOURCES;
+  kp->stages = stages;
+  kp->ring_a_off = ring_a_off;
+  kp->ring_a_bytes = ring_a_bytes;
+  kp->ring_a_geom = ring_a_bytes >= 2 * kp->slot_bytes[1] ? 1 : 0;
+  return ENTWINE_OK;
 }
 
 // Common launch path.  `partial` overrides the workspace in consumer-only mode.
@@ -1266,8 +1320,10 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   d->seq += 1;
   kp.seq = d->seq;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  ring_geometry(g, &kp);
+  rc = ring_geometry(p, &kp);
+  if (rc != ENTWINE_OK) return rc;
   kp.colocate = p->colocate;
+  kp.prefetch = p->prefetch;
   kp.out = static_cast<__nv_bfloat16*>(out);
   kp.flags_own = d->flags_own;
   kp.flags_peer = d->flags_peer;
@@ -1314,7 +1370,8 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
                      kBK, kBM, true) &&
             make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
                      kBK, (mode != MODE_COMM_ONLY) ? (pair ? 128 : g.BN) : kBM, true) &&
-            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true);
+            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
     ok = make_map(&maps.c_ld[id], c_src, g.M, g.N, kTile, rs, false) &&
@@ -1536,8 +1593,12 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  ring_geometry(g, &kp);
+  {
+    const int grc = ring_geometry(p, &kp);
+    if (grc != ENTWINE_OK) return grc;
+  }
   kp.colocate = p->colocate;
+  kp.prefetch = p->prefetch;
   kp.out = static_cast<__nv_bfloat16*>(out_shard);
   kp.status = reinterpret_cast<StatusSlot*>(ctrl + off_status);
   kp.done_ctr = reinterpret_cast<unsigned*>(ctrl + off_done);
@@ -1559,7 +1620,8 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   std::memset(&maps, 0, sizeof(maps));
   bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
             make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
-            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true);
+            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
     ok = make_map(&maps.c_ld[id], base, g.M, g.N, kTile, rs, false) &&

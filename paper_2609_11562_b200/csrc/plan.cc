@@ -248,6 +248,14 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       }
       return rc;
     }
+    case ENTWINE_OPT_STAGES:
+      if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
+      p->stages = int(value);
+      return ENTWINE_OK;
+    case ENTWINE_OPT_PREFETCH:
+      if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
+      p->prefetch = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_COLOCATE:
       if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
       p->colocate = int(value);
