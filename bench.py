@@ -32,12 +32,15 @@ METRIC = "fused GEMM-RS TFLOP/s and fraction of max(tensor peak, HBM) roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (bytes read + written per launch) of the fused kernel from an ncu capture of
 # the named workload; see profiles/.  None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"attn_out_proj": 67.22e6, "mlp_down_proj": 921.06e6, "short_k_comm_bound": 586.73e6}
 # Launch configuration per workload: communication SMs, tile order.
+# Launch configuration per workload (the best point of a budget x order scan on B200): number of
+# dedicated communication SMs (0 = consumer warps co-located with the producer in every CTA),
+# tile order (1 = interleaved, Eq. 1; 0 = row-major).
 LAUNCH = {
-    "attn_out_proj": dict(n_comm_sms=20, order=1, rank=1),
-    "mlp_down_proj": dict(n_comm_sms=20, order=1, rank=5),
-    "short_k_comm_bound": dict(n_comm_sms=16, order=1, rank=2),
+    "attn_out_proj": dict(n_comm_sms=0, order=1, rank=1),
+    "mlp_down_proj": dict(n_comm_sms=0, order=1, rank=5),
+    "short_k_comm_bound": dict(n_comm_sms=16, order=0, rank=2),
     "tiny": dict(n_comm_sms=4, order=1, rank=0),
 }
 
@@ -296,6 +299,8 @@ def main():
                          "JSON line per point to --sweep-out and print a summary line")
     ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
     ap.add_argument("--sweep-iters", type=int, default=8)
+    ap.add_argument("--comm-curve", action="store_true",
+                    help="consumer bandwidth in isolation against the number of consumer CTAs (App. A)")
     ap.add_argument("--comm-ctas", type=int, default=0,
                     help="with --kernel-only comm: number of consumer CTAs (0 = one per SM)")
     ap.add_argument("--kernel-only", default=None, choices=["fused", "gemm", "comm"],
@@ -330,6 +335,23 @@ def main():
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB of L2
     if args.sweep:
         return run_sweep(args, peaks, flush, torch, E, I)
+    if args.comm_curve:
+        # every input available, no competing producer: bandwidth against the budget (App. A)
+        A, Bm = I.make_operands(wl, device="cuda")
+        P = I.make_peer_partials(wl, device="cuda")
+        out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        curve = []
+        for x in (2, 4, 8, 12, 16, 20, 24, 32, 48, 64, 96, 128, 148):
+            plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], x if x <= 128 else 0, rank=launch["rank"])
+            plan.gemm_only(A, Bm)
+            us = statistics.median(time_steps(lambda: plan.comm_only(None, P, out, send, x), 6, 2, flush, torch))
+            plan.last_status()
+            curve.append({"consumer_ctas": x, "us": us, "GBps": wl.comm_bytes / us / 1e3,
+                          "GBps_per_cta": wl.comm_bytes / us / 1e3 / x})
+            plan.destroy()
+        print(json.dumps({"comm_curve": wl.name, "comm_bytes": wl.comm_bytes, "points": curve}))
+        return 0
     if args.kernel_only:
         A, Bm = I.make_operands(wl, device="cuda")
         P = I.make_peer_partials(wl, device="cuda")
@@ -446,7 +468,7 @@ def main():
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
     roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
-    roof["kernel"] = "entwine_fused_kernel<256>"
+    roof["kernel"] = "entwine_fused_kernel<256, true>"
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -454,7 +476,8 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K,
                    "n_comm_sms": launch["n_comm_sms"],
-                   "tile_order": "interleaved" if launch["order"] else "row_major", "block": "128x256",
+                   "tile_order": "interleaved" if launch["order"] else "row_major",
+                   "block": "128x256 blocks on CTA pairs (256x256 pair tiles)",
                    "emulated_rank": launch["rank"], "l2": "flushed between timed steps (512 MiB memset)",
                    "multi_gpu": "replicas only"},
         "us_per_call": {"mean": mean_us, "median": statistics.median(us), "min": min(us)},
@@ -487,7 +510,11 @@ def main():
                 "overlap_efficiency": med(r["gemm_only_us"]) / fused,
                 "tail_us": (r["status"]["t_end_ns"] - r["status"]["t_gemm_ns"]) / 1e3,
                 "n_comm_sms": LAUNCH[name]["n_comm_sms"],
+                "tile_order": "interleaved" if LAUNCH[name]["order"] else "row_major",
             }
+            other = dict(LAUNCH[name], order=1 - LAUNCH[name]["order"])
+            r2 = measure_workload(w2, other, max(10, args.steps // 2), 5, flush, torch, E, I, False)
+            e["other_tile_order_fused_us"] = med(r2["fused_us"])
             # Eq. 4 generalised to the emulation's push + reduce bytes, from the measured window
             t_g = r["status"]["t_gemm_ns"] * 1e-9
             if t_g > 0:

@@ -18,8 +18,8 @@ if torch.cuda.is_available():
 
 # (workload, rank, orders, budgets): the budgets are the ones the configurations name
 FULL = [
-    (I.ATTN_OUT, 1, (1, 0), (20,)),
-    (I.MLP_DOWN, 5, (1,), (20,)),
+    (I.ATTN_OUT, 1, (1, 0), (0, 20)),
+    (I.MLP_DOWN, 5, (1,), (0, 20)),
     (I.SHORT_K, 2, (1, 0), (8, 16, 24)),
 ]
 
