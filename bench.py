@@ -129,6 +129,21 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(value, dist, device):
+    """Largest per-rank value (ranks run independent replicas; the job is as slow as its slowest)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(world, flops_per_rank, seconds):
+    """Aggregate throughput of `world` replicas that each did flops_per_rank in `seconds`."""
+    return world * flops_per_rank / seconds / 1e12
+
+
 def _dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), \
         int(os.environ.get("WORLD_SIZE", "1"))
@@ -415,13 +430,9 @@ def main():
                          "timed region shorter than the sampling period: same load continued untimed")
     us = [a.elapsed_time(b) * 1e3 for a, b in evs]
     status = plan.last_status()
-    total_us = sum(us)
-    if dist is not None:
-        t = torch.tensor([total_us], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_us = float(t.item())
+    total_us = max_over_ranks(sum(us), dist, "cuda")
     mean_us = total_us / args.steps
-    value = world * wl.flops / (mean_us * 1e-6) / 1e12
+    value = whole_job_tflops(world, wl.flops, mean_us * 1e-6)
 
     # ---- end to end through the host-buffer entry point ---------------------------------------
     hA, hB, hP = A.cpu().pin_memory(), Bm.cpu().pin_memory(), P.cpu().pin_memory()
@@ -436,14 +447,10 @@ def main():
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         plan.gemm_rs_host(hA, hB, hP, hOut, hSend)
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks((time.perf_counter() - t0) / e2e_steps, dist, "cuda")
     h2d = (wl.M * wl.K + wl.N * wl.K + (wl.W - 1) * wl.R * wl.N) * 2
     d2h = (wl.R * wl.N + (wl.W - 1) * wl.R * wl.N) * 2
-    e2e = {"value": world * wl.flops / e2e_s / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+    e2e = {"value": whole_job_tflops(world, wl.flops, e2e_s), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3}
     plan.destroy()
     del hA, hB, hP, hOut, hSend, A, Bm, P, out, send
