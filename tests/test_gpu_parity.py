@@ -287,3 +287,58 @@ def test_host_buffer_entry_point():
     res = O.gemm_rs(I.bits(A), I.bits(Bm), I.bits(P), r, wl.W, 256, 1, 4)
     _check_against_oracle(wl, r, res, out, send)
     p.destroy()
+
+
+OPTION_SETS = [
+    dict(colocate=0), dict(colocate=0, tail_help=0), dict(stages=3), dict(stages=4), dict(stages=5),
+    dict(prefetch=1), dict(pair_ctas=0, stages=3), dict(tail_help=0),
+]
+
+
+@pytest.mark.parametrize("opts", OPTION_SETS, ids=lambda o: "-".join(f"{k}{v}" for k, v in o.items()))
+def test_fused_options_match_oracle(opts):
+    """Every launch option changes only how the work is scheduled on the chip: counts, the
+    oracle tolerance and bitwise equality with the default configuration must all hold."""
+    wl = SMALL[4]
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    Ad, Bd, Pd = A.cuda(), Bm.cuda(), P.cuda()
+    r = 2
+    res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, 1, 8)
+    base = None
+    for order, n_comm in itertools.product((0, 1), (0, 8)):
+        ref_plan = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=r)
+        out0, send0 = _alloc_outputs(wl)
+        ref_plan.gemm_rs(Ad, Bd, Pd, out0, send0)
+        ref_plan.last_status()
+        ref_plan.destroy()
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=r, **opts)
+        out, send = _alloc_outputs(wl)
+        for _ in range(2):
+            p.gemm_rs(Ad, Bd, Pd, out, send)
+            st = p.last_status()
+            c = p.counts()
+            assert st["flags_published"] == c["flags_published"]
+            assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+        _check_against_oracle(wl, r, res, out, send)
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        p.destroy()
+
+
+def test_many_ranks_small_steps():
+    """W = 16: the consumer's steps shrink to a few rows per contribution."""
+    wl = _small("w16", 16, 2048, 512, 256, idx=7)
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    for r, order, n_comm in ((0, 1, 0), (15, 0, 4), (7, 1, 12)):
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=r)
+        c = p.counts()
+        res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, order, c["x"])
+        out, send = _alloc_outputs(wl)
+        p.gemm_rs(A.cuda(), Bm.cuda(), P.cuda(), out, send)
+        st = p.last_status()
+        assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+        _check_against_oracle(wl, r, res, out, send)
+        p.destroy()
