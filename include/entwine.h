@@ -83,6 +83,10 @@ enum {
                                       loading half of the B panel); 0: every CTA works alone     */
   ENTWINE_OPT_PREFETCH        = 10, /* 1: the consumer's polling warp prefetches the next reduce
                                       task's published peer tiles into L2; 0 (default): off      */
+  ENTWINE_OPT_L2_HINTS        = 12, /* L2 eviction policies on TMA traffic, bit mask (default 3):
+                                      bit 0: the consumer's tile loads and pushed-tile stores are
+                                      evict-first (touched once); bit 1: the producer's operand
+                                      loads are evict-last (panels are re-read by many CTAs)     */
   ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */

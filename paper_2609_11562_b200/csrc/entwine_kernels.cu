@@ -86,6 +86,7 @@ struct KParams {
   int help;       // CTAs take tasks from lists other than their own
   int colocate;   // a producer CTA's consumer warps work while it still produces
   int prefetch;   // pull the next reduce task's peer tiles into L2 ahead of its loads
+  int l2_hints;   // consumer TMA traffic carries an evict-first L2 policy
   int stages;     // operand-ring stages of the producer
   int ring_a_off, ring_a_bytes;  // consumer ring A (after the epilogue staging)
   int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
@@ -160,6 +161,36 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// L2 eviction-priority policies for the cache-hinted TMA forms
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, int x, int y, uint32_t src,
+                                                  uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
+               ::"l"(map), "r"(x), "r"(y), "r"(src), "l"(policy)
+               : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src)
@@ -208,6 +239,14 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
       "[%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                      uint32_t bar_cluster_addr, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      ".L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
@@ -455,6 +494,8 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
 
   if (warp == kCommWarp) {
     // ---------------- claim, poll, load ----------------
+    // tiles are read once: ask L2 to evict them first so that the producer's operand panels stay
+    const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     int it = 0;
     bool ok = true;
     const long long MN = (long long)P.M * P.N, RN = P.R * (long long)P.N;
@@ -586,14 +627,14 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
             // rs rows of the local contribution first, then of the peers in ascending rank
             // order; lane q issues contribution q's load
             for (int q = lane; q < P.W; q += 32) {
-              if (q == 0) tma_load_2d(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot));
-              else tma_load_2d(dst + q * sub_bytes, &maps.p_ld[ring.geom], col, (q - 1) * P.M + src_row + step * rs,
-                               ring.full(slot));
+              if (q == 0) tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot), pol);
+              else tma_load_2d_hint(dst + q * sub_bytes, &maps.p_ld[ring.geom], col,
+                                    (q - 1) * P.M + src_row + step * rs, ring.full(slot), pol);
             }
           } else {
             for (int rr = lane * rs; rr < ring.prs; rr += 32 * rs)
-              tma_load_2d(dst + rr * kTile * 2, &maps.c_ld[ring.geom], col, src_row + step * ring.prs + rr,
-                          ring.full(slot));
+              tma_load_2d_hint(dst + rr * kTile * 2, &maps.c_ld[ring.geom], col, src_row + step * ring.prs + rr,
+                               ring.full(slot), pol);
           }
         }
         if (lane == 0) {
@@ -680,6 +721,8 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
     // which is awaited only when kPend younger stores exist or when this thread would idle.
     constexpr int kPend = 3;
+    // pushed tiles are not read again on this GPU
+    const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     unsigned long long pend = 0;  // queue of barrier addresses' slot/ring ids, 8 bits each
     int n_pend = 0;
     auto retire_all = [&]() {
@@ -717,7 +760,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
         for (int rr = 0; rr < ring.prs; rr += ring.rs)
-          tma_store_2d(&maps.send_st[ring.geom], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2);
+          tma_store_2d_hint(&maps.send_st[ring.geom], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2, pol);
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
@@ -818,6 +861,8 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 
     if (warp == kTmaWarp && lane == 0) {
       // ---- TMA producer (every CTA loads its own operands) ----
+      // operand panels are re-read by many CTAs: ask L2 to keep them
+      const uint64_t op_pol = (P.l2_hints & 2) ? l2_policy_evict_last() : l2_policy_evict_normal();
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -832,12 +877,13 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
             // both CTAs' bytes are counted on the leader's barrier, which the leader arms
             if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * C::kStageBytes);
             const uint32_t lead_bar = map_to_cta(full_bar(stage), 0);
-            tma_load_2d_pair(a_dst, &maps.a, kb * kBK, mb * kBM, lead_bar);
-            tma_load_2d_pair(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN + (int)cta_rank * C::kBRows, lead_bar);
+            tma_load_2d_pair_hint(a_dst, &maps.a, kb * kBK, mb * kBM, lead_bar, op_pol);
+            tma_load_2d_pair_hint(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN + (int)cta_rank * C::kBRows,
+                                  lead_bar, op_pol);
           } else {
             mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
-            tma_load_2d(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage));
-            tma_load_2d(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage));
+            tma_load_2d_hint(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage), op_pol);
+            tma_load_2d_hint(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage), op_pol);
           }
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
@@ -1324,6 +1370,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   if (rc != ENTWINE_OK) return rc;
   kp.colocate = p->colocate;
   kp.prefetch = p->prefetch;
+  kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out);
   kp.flags_own = d->flags_own;
   kp.flags_peer = d->flags_peer;
@@ -1599,6 +1646,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   }
   kp.colocate = p->colocate;
   kp.prefetch = p->prefetch;
+  kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out_shard);
   kp.status = reinterpret_cast<StatusSlot*>(ctrl + off_status);
   kp.done_ctr = reinterpret_cast<unsigned*>(ctrl + off_done);

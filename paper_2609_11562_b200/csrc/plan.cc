@@ -248,6 +248,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       }
       return rc;
     }
+    case ENTWINE_OPT_L2_HINTS:
+      if (value < 0 || value > 3) return ENTWINE_ERR_INVALID;
+      p->l2_hints = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_STAGES:
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);
