@@ -87,6 +87,10 @@ enum {
                                       bit 0: the consumer's tile loads and pushed-tile stores are
                                       evict-first (touched once); bit 1: the producer's operand
                                       loads are evict-last (panels are re-read by many CTAs)     */
+  ENTWINE_OPT_LISTS           = 13, /* [pre] number of consumer task lists x (Sec. 3.1: tile t of the
+                                      own partition goes to list t mod x); 0 (default): one list
+                                      per consumer CTA.  With fewer lists than CTAs the CTAs share
+                                      lists through the lists' head counters                     */
   ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */

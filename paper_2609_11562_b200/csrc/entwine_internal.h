@@ -76,6 +76,7 @@ struct Plan {
   int tail_help = 1;
   int prefetch = 0;         // look-ahead L2 prefetch of peer tiles (measured: no gain)
   int l2_hints = 3;         // bit 0: evict-first on the consumer's TMA traffic, bit 1: evict-last on operands
+  int lists_opt = 0;        // number of consumer lists x, 0 = one per consumer CTA
   int stages = 0;           // operand-ring stages of the producer, 0 = choose
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles

@@ -1360,7 +1360,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.cpb = g.cpb; kp.R = g.R;
   kp.x = p->x;
   kp.mode = mode;
-  kp.help = p->tail_help;
+  kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = (mode == MODE_COMM_ONLY) ? 1 : 0;
   kp.epoch = d->epoch;
   d->seq += 1;
@@ -1635,7 +1635,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.cpb = g.cpb; kp.R = g.R;
   kp.x = p->x;
   kp.mode = MODE_FUSED;
-  kp.help = p->tail_help;
+  kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = 0;
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;

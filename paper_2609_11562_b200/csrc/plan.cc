@@ -165,6 +165,7 @@ int finalize_plan(Plan* p) {
     if (p->n_gemm_ctas < 1) return ENTWINE_ERR_INVALID;
     p->x = p->n_comm_sms;
   }
+  if (p->lists_opt > 0) p->x = p->lists_opt;
   build_tables(p->g, p->order, p->rank, p->x, p->n_gemm_ctas, p->n_comm_ctas, &p->tables);
   p->tables_built = true;
   return ENTWINE_OK;
@@ -252,6 +253,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       if (value < 0 || value > 3) return ENTWINE_ERR_INVALID;
       p->l2_hints = int(value);
       return ENTWINE_OK;
+    case ENTWINE_OPT_LISTS:
+      if (p->launched || value < 0 || value > 4096) return ENTWINE_ERR_INVALID;
+      p->lists_opt = int(value);
+      return entwine::finalize_plan(p);
     case ENTWINE_OPT_STAGES:
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);

@@ -102,6 +102,19 @@ def test_exported_tables_equal_oracle(M, N, K, W):
         p.destroy()
 
 
+def test_list_count_option_follows_the_oracle():
+    """x (the number of consumer lists) can be set apart from the number of consumer CTAs."""
+    M, N, K, W, r = 2048, 1280, 64, 4, 3
+    for order, x in itertools.product((0, 1), (1, 5, 40)):
+        p = E.Plan(M, N, K, W, order, 8, num_sms=148, rank=r, lists=x)
+        assert p.counts()["x"] == x
+        s = O.schedule(M, N, W, 256, order)
+        table, offs, peer_offs = O.index_maps(s, r, x)
+        assert (p.export(E.EXPORT_LIST_OFFS) == offs).all()
+        assert (p.export(E.EXPORT_TASKS).reshape(-1, 8) == table).all()
+        p.destroy()
+
+
 def test_fig3_example_through_the_library(golden):
     g = golden("fig3_example.txt")
     W, BN, M, N = (int(g[k][0][0]) for k in ("W", "BN", "M", "N"))
