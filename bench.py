@@ -202,15 +202,17 @@ def main_reference(args, wl, launch):
     return 0
 
 
-def time_steps(fn, steps, warmup, flush, torch):
-    """Device time of `steps` calls of fn with the L2 flushed before each; returns µs list."""
+def time_steps(fn, steps, warmup, flush, torch, cold=True):
+    """Device time of `steps` calls of fn with the L2 flushed before each (cold) or not; µs list."""
     for _ in range(warmup):
-        flush.zero_()
+        if cold:
+            flush.zero_()
         fn()
     torch.cuda.synchronize()
     evs = []
     for _ in range(steps):
-        flush.zero_()
+        if cold:
+            flush.zero_()
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -233,6 +235,8 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     st = plan.last_status()
     res["fused_us"] = us
     res["status"] = st
+    res["fused_hot_us"] = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), steps, 3, flush, torch, cold=False)
+    plan.last_status()
     if detailed:
         # the producer alone (uncontended GEMM time) and the consumer alone
         res["gemm_only_us"] = time_steps(lambda: plan.gemm_only(A, Bm), max(5, steps // 4), 3, flush, torch)
@@ -506,6 +510,7 @@ def main():
             tc, hb = roofline_seconds(w2, peaks)
             e = {
                 "fused_us": fused, "fused_tflops": w2.flops / fused / 1e6,
+                "fused_hot_l2_us": med(r["fused_hot_us"]),
                 "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
                 "bound": "tensor" if tc >= hb else "hbm",
                 "unfused_cublas_then_reduce_us": med(r["unfused_us"]),
