@@ -1240,7 +1240,12 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 template <int BN, bool PAIR>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
-  static bool configured = false;
+  // per device: the shared-memory opt-in has been set, and how many clusters fit at once
+  static int max_clusters[64] = {0};
+  static bool configured[64] = {false};
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return ENTWINE_ERR_RESOURCES;
   auto kern = entwine_fused_kernel<BN, PAIR>;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
@@ -1255,20 +1260,17 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (!configured) {
+  if (!configured[dev]) {
     CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     int per_sm = 0;
     CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
     if (per_sm < 1) return ENTWINE_ERR_RESOURCES;
-    if (PAIR) {
-      // every cluster of the grid must be resident at once: producers and consumers wait on
-      // each other inside one launch
-      int clusters = 0;
-      CK(cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg));
-      if (clusters * 2 < grid) return ENTWINE_ERR_RESOURCES;
-    }
-    configured = true;
+    if (PAIR) CK(cudaOccupancyMaxActiveClusters(&max_clusters[dev], kern, &cfg));
+    configured[dev] = true;
   }
+  // every cluster of the grid must be resident at once: producers and consumers wait on each
+  // other inside one launch
+  if (PAIR && max_clusters[dev] * 2 < grid) return ENTWINE_ERR_RESOURCES;
   CK(cudaLaunchKernelEx(&cfg, kern, maps, kp));
   CK(cudaGetLastError());
   return ENTWINE_OK;
