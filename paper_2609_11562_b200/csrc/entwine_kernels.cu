@@ -115,9 +115,11 @@ struct KMaps {
   CUtensorMap a, b;      // operands
   CUtensorMap c_st;      // partial C, box 64 x 32, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
-  CUtensorMap c_ld[2];      // partial C as the consumer reads it
-  CUtensorMap p_ld[2];      // incoming partials viewed as [(W-1)*M, N]
-  CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N]
+  CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
+  CUtensorMap p_ld[2];      // incoming partials as a 3-D tensor [W-1][M][N], box 128 x rs x (W-1):
+                            // one load brings all peers' rows of a reduce step
+  CUtensorMap c_push[2];    // partial C, box 128 x prs: one load per push step
+  CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N], box 128 x prs: one store per push step
   CUtensorMap p_pf;         // incoming partials, whole-tile box, for L2 prefetch
 };
 
@@ -183,6 +185,14 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
       "[%0], [%1, {%2, %3}], [%4], %5;"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                                 uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, int x, int y, uint32_t src,
@@ -623,18 +633,16 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
           }
           ok = __all_sync(0xffffffffu, free_slot);
           if (!ok) break;
+          // Few, large TMA operations: the per-operation cost of the TMA unit, not bandwidth,
+          // bounds a consumer that issues many small boxes.
           if (task.kind == 0) {
-            // rs rows of the local contribution first, then of the peers in ascending rank
-            // order; lane q issues contribution q's load
-            for (int q = lane; q < P.W; q += 32) {
-              if (q == 0) tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot), pol);
-              else tma_load_2d_hint(dst + q * sub_bytes, &maps.p_ld[ring.geom], col,
-                                    (q - 1) * P.M + src_row + step * rs, ring.full(slot), pol);
-            }
-          } else {
-            for (int rr = lane * rs; rr < ring.prs; rr += 32 * rs)
-              tma_load_2d_hint(dst + rr * kTile * 2, &maps.c_ld[ring.geom], col, src_row + step * ring.prs + rr,
-                               ring.full(slot), pol);
+            // rs rows of the local contribution (lane 0), then of all peers in ascending rank
+            // order as one 3-D box (lane 1)
+            if (lane == 0) tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot), pol);
+            if (lane == 1)
+              tma_load_3d_hint(dst + sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rs, 0, ring.full(slot), pol);
+          } else if (lane == 0) {
+            tma_load_2d_hint(dst, &maps.c_push[ring.geom], col, src_row + step * ring.prs, ring.full(slot), pol);
           }
         }
         if (lane == 0) {
@@ -759,8 +767,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       if (m.kind == 0) {
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
-        for (int rr = 0; rr < ring.prs; rr += ring.rs)
-          tma_store_2d_hint(&maps.send_st[ring.geom], m.dst_x, m.dst_y + rr, sbase + rr * kTile * 2, pol);
+        tma_store_2d_hint(&maps.send_st[ring.geom], m.dst_x, m.dst_y, sbase, pol);
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
@@ -1142,6 +1149,21 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
   return rc == CUDA_SUCCESS;
 }
 
+// 3-D map over bf16 [planes][rows][cols] with a (box_planes x box_rows x box_cols) box, no swizzle.
+static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_t rows, int64_t cols,
+                      int box_cols, int box_rows, int box_planes) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), cuuint64_t(planes)};
+  cuuint64_t strides[2] = {cuuint64_t(cols) * 2, cuuint64_t(cols) * cuuint64_t(rows) * 2};
+  cuuint32_t box[3] = {cuuint32_t(box_cols), cuuint32_t(box_rows), cuuint32_t(box_planes)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS;
+}
+
 int device_sm_count() {
   int n = 0;
   if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) {
@@ -1423,9 +1445,12 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
             make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
+    const int prs = kp.prs[id];
     ok = make_map(&maps.c_ld[id], c_src, g.M, g.N, kTile, rs, false) &&
-         make_map(&maps.p_ld[id], comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, rs, false) &&
-         make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, rs, false);
+         make_map(&maps.c_push[id], c_src, g.M, g.N, kTile, prs, false) &&
+         (comm ? make_map3(&maps.p_ld[id], peers, g.W - 1, g.M, g.N, kTile, rs, g.W - 1)
+               : make_map3(&maps.p_ld[id], d->C, 1, g.M, g.N, kTile, rs, 1)) &&
+         make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, prs, false);
   }
   if (!ok) return ENTWINE_ERR_CUDA;
   if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
@@ -1674,9 +1699,11 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
             make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
+    const int prs = kp.prs[id];
     ok = make_map(&maps.c_ld[id], base, g.M, g.N, kTile, rs, false) &&
-         make_map(&maps.p_ld[id], peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, rs, false) &&
-         make_map(&maps.send_st[id], send_bufs, int64_t(g.W - 1) * g.R, g.N, kTile, rs, false);
+         make_map(&maps.c_push[id], base, g.M, g.N, kTile, prs, false) &&
+         make_map3(&maps.p_ld[id], peer_partials, g.W - 1, g.M, g.N, kTile, rs, g.W - 1) &&
+         make_map(&maps.send_st[id], send_bufs, int64_t(g.W - 1) * g.R, g.N, kTile, prs, false);
   }
   if (!ok) return ENTWINE_ERR_CUDA;
   int rc;
