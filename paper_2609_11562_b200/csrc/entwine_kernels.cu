@@ -23,7 +23,7 @@ constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
 // Warp roles of the 16 warps of a CTA.  Producer work (warps 0, 1, 4-7) and consumer work
 // (warps 2, 3, 8-15) run side by side in a producer CTA: the tensor pipe is driven by one
 // thread, so the SM's TMA and ALUs are free to move and reduce tiles meanwhile.
-constexpr int kThreads = 512;
+constexpr int kThreads = 576;
 constexpr int kTmaWarp = 0;       // producer: TMA loads of A and B
 constexpr int kMmaWarp = 1;       // producer: tcgen05.mma issue, TMEM owner
 constexpr int kCommWarp = 2;      // consumer: claims tasks, polls flags, issues TMA loads
@@ -32,21 +32,23 @@ constexpr int kEpiWarp0 = 4;      // producer: epilogue warps 4..7
 constexpr int kEpiThreads = 128;
 constexpr int kRedWarp0 = 8;      // consumer: reducing warps 8..15
 constexpr int kRedThreads = 256;
-constexpr int kGemmThreads = 192; // warps 0, 1, 4-7
+constexpr int kCStoreWarp = 16;   // producer: TMA stores of the partial C
+constexpr int kFlagWarp = 17;     // producer: releases the tile flags of stored blocks
+constexpr int kGemmThreads = 256; // warps 0, 1, 4-7, 16, 17
 constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abort flag
-constexpr int kEpiStageBytes = 8192;  // per epilogue warp: 32 rows x 128 columns of bf16
+constexpr int kEpiBufBytes = 16384;   // one staging buffer: 128 rows x 64 columns of bf16, 128B-swizzled
 
 // Shared-memory map (offsets from a 1024-byte aligned base).  The first 224 KiB are split at
 // launch time between the producer's operand ring (S stages), the epilogue staging and the
 // consumer's ring A, which a producer CTA's consumer warps use while it still produces:
 //   [0, S*stage)                operand ring of the producer
-//   [S*stage, S*stage + 32 KiB) epilogue staging (4 x 8 KiB)
+//   [S*stage, S*stage + 32 KiB) epilogue staging (2 x 16 KiB)
 //   [.., 229376)                consumer ring A (32 KiB with 5 pair stages, 64 KiB with 4, ...)
 //   [0, 196608)                 consumer ring B: 6 slots of 32 KiB, used once the CTA's producer
 //                               work is over (and by dedicated consumer CTAs from the start)
 //   [229376, 230016)            mbarriers, TMEM base slot
 constexpr int kDataBytes = 229376;
-constexpr int kStagingBytes = 4 * kEpiStageBytes;
+constexpr int kStagingBytes = 2 * kEpiBufBytes;
 constexpr int kRingBOff = 0;
 constexpr int kRingBBytes = 196608;
 constexpr int kMaxSlots = 8;
@@ -56,6 +58,7 @@ constexpr int kBarBytes = 640;
 constexpr int kBarGemm = 0;        // full[6], empty[6], tfull[2], tempty[2]
 constexpr int kBarTmemSlot = 136;
 constexpr int kBarPair = 144;      // end-of-producer handshake of a CTA pair
+constexpr int kBarStaging = 152;   // staged[2], free[2]: epilogue warps <-> publishing warp
 constexpr int kBarRingA = 192;     // full[8], empty[8], reduced[8]
 constexpr int kBarRingB = 192 + 192;
 constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
@@ -91,6 +94,7 @@ struct KParams {
   int ring_a_off, ring_a_bytes;  // consumer ring A (after the epilogue staging)
   int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
   int skip_wait;  // treat every flag as published (consumer in isolation)
+  int claim;      // most consecutive tasks taken from a list per claim
   // consumer ring geometry, [0] ring A (small, beside the producer's buffers), [1] ring B
   int rs[2];         // rows of a tile moved per reduce step (all W contributions of those rows)
   int prs[2];        // rows of a tile moved per push step
@@ -113,7 +117,7 @@ struct KParams {
 // 128-byte swizzle; the consumer's maps are plain row-major boxes of 128 columns x rs rows.
 struct KMaps {
   CUtensorMap a, b;      // operands
-  CUtensorMap c_st;      // partial C, box 64 x 32, swizzled (epilogue stores)
+  CUtensorMap c_st;      // partial C, box 64 x 128, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
   CUtensorMap p_ld[2];      // incoming partials as a 3-D tensor [W-1][M][N], box 128 x rs x (W-1):
@@ -332,10 +336,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ unsigned ld_relaxed_gpu(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+__device__ __forceinline__ void st_release_cta(int* p, int v) {
+  asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const int* p) {
+  int v;
+  asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+__device__ __forceinline__ void st_relaxed_gpu(unsigned* p, unsigned v) {
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void st_release_gpu(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -393,6 +414,7 @@ struct SlotMeta {
 struct CtaShared {
   volatile int abort;      // a role of this CTA (or another CTA) gave up
   volatile int gemm_done;  // this CTA's producer work is over; its shared memory is free
+  int blocks_stored;       // blocks of this CTA whose partial-C stores are complete
   SlotMeta meta[2][kMaxSlots];
 };
 
@@ -518,9 +540,16 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       if (!done) return;
       bool free_slot = true;
       if (lane == 0) {
-        const int slot = it % ring.n_slots;
-        free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+        // Ring B overlaps ring A's memory: every step still in flight in ring A must have been
+        // reduced or forwarded (its slot returned) before ring B is loaded.  Slot s has been
+        // used uses(s) times; its last use, number uses(s) - 1, is over when the empty barrier
+        // completes the phase of that parity.
+        for (int sl = 0; free_slot && sl < ring.n_slots; ++sl) {
+          const int uses = (it - sl + ring.n_slots - 1) / ring.n_slots;
+          if (uses > 0) free_slot = mbar_wait(ring.empty(sl), (uses - 1) & 1, P, sh);
+        }
         if (free_slot) {
+          const int slot = it % ring.n_slots;
           sh->meta[0][slot].kind = -2;
           mbar_arrive(ring.full(slot));
         }
@@ -529,127 +558,190 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       ring = make_ring(smem_base, 1, P);
       it = 0;
     };
-    // Drains list j: claims go through the list's head counter, so the list is consumed in
-    // order whoever executes it.  Two claims are kept in flight to hide the atomics' latency;
-    // a window of 32 task records (one per lane) is refilled when a claim falls outside it.
+    // Drains list j.  Claims go through the list's head counter in runs of up to P.claim
+    // consecutive tasks, so the list is consumed in order whoever executes it (Sec. 3.1).  This
+    // warp is the one serial stage of the pipeline and a push task is a single ring step, so the
+    // per-task path is kept short:
+    //   * nothing a task needs from global memory is waited for on that path: three claims are
+    //     kept going (`cur` is executed, `nxt` has its flags in flight, `fut` its atomic), a
+    //     window of 32 task records is loaded ahead of the first claim's return, and the flags
+    //     of claim `nxt` are read early with relaxed loads (up to 64 flags, two per lane); when
+    //     `nxt` becomes `cur`, flags seen as published are made an acquire by one fence for the
+    //     whole claim, the others fall back to the acquire poll of Sec. 4.2;
+    //   * the 32 lanes turn the 32 records of a window into load coordinates in parallel
+    //     (checks, divisions), and one lane then runs a task's ring steps without warp votes.
     auto drain = [&](int j) {
       const int base = P.list_offs[j];
       const int len = P.list_offs[j + 1] - base;
-      int c0 = len, c1 = len;
+      if (len <= 0) return;
+      const int CH = P.claim;  // CH * W <= 64 (W <= 64): the flags of a claim fit the early look
+      // Claims shrink towards the end of the list (guided self-scheduling) so that the CTAs that
+      // share it finish together: a quarter of an even share of what is left, at most CH tasks.
+      const int sharers = ((int)gridDim.x + P.x - 1) / P.x;
+      auto claim_len = [&](int head) { return max(1, min(CH, (len - head) / (4 * sharers))); };
+      int cur = len, nxt = len, fut = len;
+      int cur_n = claim_len(0), nxt_n = cur_n, fut_n = cur_n;
       if (lane == 0) {
-        c0 = atomicAdd(&P.list_head[j], 1);
-        c1 = atomicAdd(&P.list_head[j], 1);
+        cur = atomicAdd(&P.list_head[j], cur_n);
+        nxt = atomicAdd(&P.list_head[j], nxt_n);
+        fut = atomicAdd(&P.list_head[j], fut_n);
       }
-      int win = -(1 << 30);
-      Task mine;
-      mine.kind = 0; mine.d = 0; mine.t = 0; mine.slot = 0; mine.src_off = 0; mine.dst_off = 0;
+      // this lane's record of the window, as coordinates: kind (-3 = record out of range), tile
+      // column, row of the tile in an [M,N] buffer, first destination row, flag indices
+      int win = 0;
+      int k_kind, k_col, k_row, k_dst, k_own, k_t;
+      auto load_window = [&](int first) {
+        win = first;
+        const Task rec = P.tasks[base + min(first + lane, len - 1)];
+        const bool bad = rec.src_off < 0 || rec.src_off + (long long)(kTile - 1) * P.N + kTile > MN ||
+                         rec.dst_off < 0 || rec.dst_off + (long long)(kTile - 1) * P.N + kTile > RN ||
+                         rec.t < 0 || rec.t >= P.Q || rec.d < 0 || rec.d >= P.W ||
+                         (rec.kind == 1 && (rec.slot < 0 || rec.slot >= P.W - 1));
+        const int trow = rec.t / P.nTn, tcol = rec.t - trow * P.nTn;
+        k_kind = bad ? -3 : rec.kind;
+        k_col = tcol * kTile;
+        k_row = rec.d * (int)P.R + trow * kTile;
+        k_dst = (rec.kind == 0 ? 0 : rec.slot * (int)P.R) + trow * kTile;
+        k_own = rec.d * P.Q + rec.t;
+        k_t = rec.t;
+      };
+      load_window(0);
+      unsigned pf[2] = {0u, 0u};
+      int pf_start = -1;
+      // relaxed look at the flags of the claim starting at s (if its records are in the window)
+      auto peek_flags = [&](int s, int n_claim) {
+        pf_start = -1;
+        if (P.skip_wait || s >= len || s < win || s + n_claim > win + 32) return;
+        pf_start = s;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int f = r * 32 + lane;
+          const int c = f / P.W, q = f - c * P.W;
+          const int src = min(s - win + c, 31);
+          const int kind = __shfl_sync(0xffffffffu, k_kind, src);
+          const int own = __shfl_sync(0xffffffffu, k_own, src);
+          const int t = __shfl_sync(0xffffffffu, k_t, src);
+          pf[r] = 0xffffffffu;
+          if (c < n_claim && s + c < len && kind >= 0) {
+            if (q == 0) pf[r] = ld_relaxed_gpu(&P.flags_own[own]);
+            else if (kind == 0) pf[r] = ld_relaxed_gpu(&P.flags_peer[(q - 1) * P.Q + t]);
+          }
+        }
+      };
       while (ok) {
-        const int i = __shfl_sync(0xffffffffu, c0, 0);
-        if (i >= len) break;
-        c0 = c1;
-        if (lane == 0) c1 = atomicAdd(&P.list_head[j], 1);
-        if (i < win || i >= win + 32) {
-          win = i;
-          mine = P.tasks[base + min(i + lane, len - 1)];
+        const int s = __shfl_sync(0xffffffffu, cur, 0);
+        if (s >= len) break;
+        const int n = min(cur_n, len - s);
+        // tasks of this claim whose flags were all seen as published by the early look
+        unsigned ready = 0;
+        if (pf_start == s) {
+          unsigned unset = 0;
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int c = (r * 32 + lane) / P.W;
+            if (pf[r] < P.epoch) unset |= 1u << min(c, 31);
+          }
+          ready = ~__reduce_or_sync(0xffffffffu, unset) & ((1u << n) - 1u);
+          if (ready) {
+            fence_acq_rel_gpu();  // relaxed reads of published flags + this fence = acquire
+            fence_async_all();    // and the TMA reads below are ordered after it
+          }
         }
-        const int src = i - win;
-        Task task;
-        task.kind = __shfl_sync(0xffffffffu, mine.kind, src);
-        task.d = __shfl_sync(0xffffffffu, mine.d, src);
-        task.t = __shfl_sync(0xffffffffu, mine.t, src);
-        task.slot = __shfl_sync(0xffffffffu, mine.slot, src);
-        task.src_off = __shfl_sync(0xffffffffu, mine.src_off, src);
-        task.dst_off = __shfl_sync(0xffffffffu, mine.dst_off, src);
-        // index check: record and skip instead of touching memory out of range
-        const bool bad = task.src_off < 0 || task.src_off + (long long)(kTile - 1) * P.N + kTile > MN ||
-                         task.dst_off < 0 || task.dst_off + (long long)(kTile - 1) * P.N + kTile > RN ||
-                         task.t < 0 || task.t >= P.Q || task.d < 0 || task.d >= P.W ||
-                         (task.kind == 1 && (task.slot < 0 || task.slot >= P.W - 1));
-        if (bad) {
-          if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
-          continue;
-        }
-        if (P.prefetch) {
-          // Look-ahead: the claim after this one names the next task.  If it is a reduce task
-          // whose peer contributions are already published, pull their tiles into L2 now (one
-          // lane per peer) so that the ring's loads find them there while holding a slot.
-          const int nx = __shfl_sync(0xffffffffu, c0, 0);
-          if (nx < len && nx >= win && nx < win + 32) {
-            const int lk = nx - win;
-            const int nkind = __shfl_sync(0xffffffffu, mine.kind, lk);
-            const int nd = __shfl_sync(0xffffffffu, mine.d, lk);
-            const int nt = __shfl_sync(0xffffffffu, mine.t, lk);
-            if (nkind == 0 && nt >= 0 && nt < P.Q && nd >= 0 && nd < P.W) {
-              const int nrow = nd * (int)P.R + (nt / P.nTn) * kTile, ncol = (nt % P.nTn) * kTile;
+        // rotate the claims (after the fence, which waits for the atomics in flight)
+        cur = nxt;
+        nxt = fut;
+        cur_n = nxt_n;
+        nxt_n = fut_n;
+        fut_n = claim_len(s + n);
+        if (lane == 0) fut = atomicAdd(&P.list_head[j], fut_n);
+        if (s < win || s + n > win + 32) load_window(s);
+        peek_flags(__shfl_sync(0xffffffffu, cur, 0), cur_n);
+        for (int c = 0; ok && c < n; ++c) {
+          const int i = s + c;
+          const int src = i - win;
+          const int kind = __shfl_sync(0xffffffffu, k_kind, src);
+          const int col = __shfl_sync(0xffffffffu, k_col, src);
+          const int src_row = __shfl_sync(0xffffffffu, k_row, src);
+          const int dst_row = __shfl_sync(0xffffffffu, k_dst, src);
+          if (kind < 0) {
+            // index check failed: record and skip instead of touching memory out of range
+            if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
+            continue;
+          }
+          if (P.prefetch && c + 1 < n) {
+            // Look-ahead: if the next task of the claim is a reduce task whose peer contributions
+            // are already published, pull their tiles into L2 now (one lane per peer) so that the
+            // ring's loads find them there while holding a slot.
+            const int nkind = __shfl_sync(0xffffffffu, k_kind, src + 1);
+            const int nt = __shfl_sync(0xffffffffu, k_t, src + 1);
+            const int nrow = __shfl_sync(0xffffffffu, k_row, src + 1);
+            const int ncol = __shfl_sync(0xffffffffu, k_col, src + 1);
+            if (nkind == 0) {
               for (int q = lane - 1; q >= 0 && q < P.W - 1; q += 31) {
                 if (P.skip_wait || ld_acquire_gpu(&P.flags_peer[q * P.Q + nt]) >= P.epoch)
                   tma_prefetch_l2_2d(&maps.p_pf, ncol, q * P.M + nrow);
               }
             }
           }
-        }
-        if (!P.skip_wait) {
-          // lane 0 polls the local flag, lanes 1.. the peers' flags in rank order (Sec. 4.2);
-          // the warp proceeds when all W contributions of the tile are published
-          bool mine_ok = true;
-          if (lane == 0) mine_ok = wait_flag(&P.flags_own[task.d * P.Q + task.t], P);
-          else if (task.kind == 0) {
-            for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
-              mine_ok = wait_flag(&P.flags_peer[q * P.Q + task.t], P);
+          if (!P.skip_wait && !((ready >> c) & 1u)) {
+            // lane 0 polls the local flag, lanes 1.. the peers' flags in rank order (Sec. 4.2);
+            // the warp proceeds when all W contributions of the tile are published
+            const int own = __shfl_sync(0xffffffffu, k_own, src);
+            const int t = __shfl_sync(0xffffffffu, k_t, src);
+            bool mine_ok = true;
+            if (lane == 0) mine_ok = wait_flag(&P.flags_own[own], P);
+            else if (kind == 0) {
+              for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
+                mine_ok = wait_flag(&P.flags_peer[q * P.Q + t], P);
+            }
+            ok = __all_sync(0xffffffffu, mine_ok);
+            if (!ok) {
+              if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
+              break;
+            }
+            fence_async_all();  // the TMA reads below are ordered after the acquires
           }
-          ok = __all_sync(0xffffffffu, mine_ok);
-          if (!ok) {
-            if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
-            break;
-          }
-          fence_async_all();  // the TMA reads below are ordered after the acquires
-        }
-        maybe_switch();
-        if (!ok) break;
-        const int trow = task.t / P.nTn, tcol = task.t % P.nTn;
-        const int col = tcol * kTile;
-        const int src_row = task.d * (int)P.R + trow * kTile;  // row of the tile in an [M,N] buffer
-        const int n_steps = kTile / (task.kind == 0 ? ring.rs : ring.prs);
-        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
-        for (int step = 0; ok && step < n_steps; ++step, ++it) {
-          const int slot = it % ring.n_slots;
-          const uint32_t ph = (it / ring.n_slots) & 1;
-          const uint32_t dst = ring.base + slot * ring.slot_bytes;
-          bool free_slot = true;
+          maybe_switch();
+          if (!ok) break;
+          const int rows = kind == 0 ? ring.rs : ring.prs;  // rows of the tile per ring step
+          const int n_steps = kTile / rows;
+          bool steps_ok = true;
           if (lane == 0) {
-            free_slot = mbar_wait(ring.empty(slot), ph ^ 1, P, sh);
-            if (free_slot) {
+            // one lane runs the task's steps: wait for the slot, describe it, issue its loads
+            int slot = it % ring.n_slots;
+            uint32_t ph = (it / ring.n_slots) & 1;
+            const uint32_t tx = kind == 0 ? P.W * ring.sub_bytes : ring.prs * kTile * 2;
+            for (int step = 0; step < n_steps; ++step) {
+              if (!mbar_wait(ring.empty(slot), ph ^ 1, P, sh)) { steps_ok = false; break; }
+              const uint32_t dst = ring.base + slot * ring.slot_bytes;
               SlotMeta& m = sh->meta[ring.id][slot];
-              m.kind = task.kind;
+              m.kind = kind;
               m.dst_x = col;
-              if (task.kind == 0) {
-                m.dst_y = trow * kTile + step * rs;
-                mbar_arrive_expect_tx(ring.full(slot), P.W * sub_bytes);
+              m.dst_y = dst_row + step * rows;
+              mbar_arrive_expect_tx(ring.full(slot), tx);
+              // Few, large TMA operations: the per-operation cost of the TMA unit, not bandwidth,
+              // bounds a consumer that issues many small boxes.
+              if (kind == 0) {
+                // rs rows of the local contribution, then of all peers in ascending rank order
+                // as one 3-D box
+                tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
+                tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
+                                 ring.full(slot), pol);
               } else {
-                m.dst_y = task.slot * (int)P.R + trow * kTile + step * ring.prs;
-                mbar_arrive_expect_tx(ring.full(slot), ring.prs * kTile * 2);
+                tma_load_2d_hint(dst, &maps.c_push[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
               }
+              if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
+            }
+            if (steps_ok) {
+              if (kind == 0) cnt->reduced++;
+              else cnt->pushed++;
+            } else {
+              report(P, -ENTWINE_ERR_TIMEOUT, base + i);
             }
           }
-          ok = __all_sync(0xffffffffu, free_slot);
-          if (!ok) break;
-          // Few, large TMA operations: the per-operation cost of the TMA unit, not bandwidth,
-          // bounds a consumer that issues many small boxes.
-          if (task.kind == 0) {
-            // rs rows of the local contribution (lane 0), then of all peers in ascending rank
-            // order as one 3-D box (lane 1)
-            if (lane == 0) tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rs, ring.full(slot), pol);
-            if (lane == 1)
-              tma_load_3d_hint(dst + sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rs, 0, ring.full(slot), pol);
-          } else if (lane == 0) {
-            tma_load_2d_hint(dst, &maps.c_push[ring.geom], col, src_row + step * ring.prs, ring.full(slot), pol);
-          }
+          ok = __all_sync(0xffffffffu, steps_ok);
+          it += n_steps;
         }
-        if (lane == 0) {
-          if (task.kind == 0) cnt->reduced++;
-          else cnt->pushed++;
-        }
-        if (!ok && lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
       }
     };
     // the CTA's own list first
@@ -687,9 +779,10 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
   } else if (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32) {
     // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
     const int ctid = threadIdx.x - kRedWarp0 * 32;
-    for (int it = 0;; ++it) {
-      const int slot = it % ring.n_slots;
-      const uint32_t ph = (it / ring.n_slots) & 1;
+    int slot = -1;
+    uint32_t ph = 0;
+    for (;;) {
+      if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
       // one lane per warp polls; the warp-level vote carries the barrier's acquire to all lanes
       bool landed = true;
       if (lane == 0) landed = mbar_wait(ring.full(slot), ph, P, sh);
@@ -701,7 +794,8 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       if (m.kind == -1) break;
       if (m.kind == -2) {
         ring = make_ring(smem_base, 1, P);
-        it = -1;
+        slot = -1;
+        ph = 0;
         continue;
       }
       if (m.kind == 0) {
@@ -741,9 +835,10 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         mbar_arrive(rr.empty(int(pend & 15u)));
       }
     };
-    for (int it = 0;; ++it) {
-      const int slot = it % ring.n_slots;
-      const uint32_t ph = (it / ring.n_slots) & 1;
+    int slot = -1;
+    uint32_t ph = 0;
+    for (;;) {
+      if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
       if (!mbar_try_wait(ring.full(slot), ph)) {
         retire_all();  // nothing to do yet: let the stores in flight return their slots
         if (!mbar_wait(ring.full(slot), ph, P, sh)) {
@@ -756,7 +851,8 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       if (m.kind == -2) {
         retire_all();
         ring = make_ring(smem_base, 1, P);
-        it = -1;
+        slot = -1;
+        ph = 0;
         continue;
       }
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
@@ -805,6 +901,8 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   const int n_stages = P.stages;
   const uint32_t tmem_slot = smem_base + kBarOff + kBarTmemSlot;
   const uint32_t pair_bar = smem_base + kBarOff + kBarPair;
+  auto staged_bar = [&](int b) { return smem_base + kBarOff + kBarStaging + 8u * b; };
+  auto sfree_bar = [&](int b) { return smem_base + kBarOff + kBarStaging + 8u * (2 + b); };
   const bool is_producer = (int)blockIdx.x < P.G && P.mode != MODE_COMM_ONLY;
   const int g = (int)blockIdx.x;                 // producer index
   const int cidx = (int)blockIdx.x - P.G;        // consumer index of a dedicated consumer CTA
@@ -818,6 +916,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 
   if (threadIdx.x == 0) {
     sh.abort = 0;
+    sh.blocks_stored = 0;
     sh.gemm_done = (is_producer && n_my > 0) ? 0 : 1;
     atomicMin(&st->t_start, globaltimer_ns());
     if (is_producer) {
@@ -830,6 +929,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * (kEpiThreads / 32));
       }
       mbar_init(pair_bar, 1);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(staged_bar(b), kEpiThreads / 32);
+        mbar_init(sfree_bar(b), 1);
+      }
     }
     for (int ring = 0; ring < 2; ++ring) {  // consumer rings: full, empty, reduced
       const uint32_t rb = smem_base + kBarOff + (ring == 0 ? kBarRingA : kBarRingB);
@@ -852,8 +955,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 
   CommCounters cnt;
   unsigned published = 0;
-  const bool gemm_warp = warp == kTmaWarp || warp == kMmaWarp || (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4);
-  const bool comm_warp = warp == kCommWarp || warp == kStoreWarp || warp >= kRedWarp0;
+  const bool gemm_warp = warp == kTmaWarp || warp == kMmaWarp || warp == kCStoreWarp || warp == kFlagWarp ||
+                         (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4);
+  const bool comm_warp = warp == kCommWarp || warp == kStoreWarp ||
+                         (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32);
 
   if (is_producer && gemm_warp) {
     // ---------------- producer: tcgen05 GEMM ----------------
@@ -931,33 +1036,36 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -2); }
-    } else if (warp >= kEpiWarp0) {
-      // ---- epilogue: TMEM -> bf16 -> swizzled staging -> TMA store of the partial C, then the
-      //      block's tile flags ----
+    } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
+      // ---- epilogue: TMEM -> bf16 -> swizzled staging.  The block leaves as BN/64 boxes of
+      //      128 rows x 64 columns through two staging buffers; the publishing warp stores them,
+      //      so these warps never wait for global memory ----
       const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
-      const uint32_t stg = smem_base + n_stages * C::kStageBytes + q * kEpiStageBytes;
+      const uint32_t stg0 = smem_base + n_stages * C::kStageBytes + (q * 32 + lane) * 128;
       int acc = 0;
       uint32_t acc_phase = 0;
+      int nbox = 0;  // boxes staged so far: buffer nbox & 1, use (nbox >> 1)
       bool ok = true;
       for (int i = 0; ok && i < n_my; ++i) {
-        int d, l;
-        block_of(i, &d, &l);
-        const int trow = l / P.nBn, nb = l % P.nBn;
-        const int mb = d * P.rowsT + trow;
         ok = mbar_wait(tfull_bar(acc), acc_phase, P, &sh);
         ok = __all_sync(0xffffffffu, ok);  // reconverge; the warp leaves the loop together
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + acc * BN;
 #pragma unroll 1
-        for (int h = 0; h < BN / kTile; ++h) {
-          // one 128-column reduction tile: 32 rows x 256 bytes per warp, as two swizzled boxes
+        for (int j = 0; j < BN / 64; ++j, ++nbox) {
+          const int buf = nbox & 1;
+          bool free_buf = true;
+          if (lane == 0) free_buf = mbar_wait(sfree_bar(buf), ((nbox >> 1) & 1) ^ 1, P, &sh);
+          ok = __all_sync(0xffffffffu, free_buf);
+          if (!ok) break;
+          const uint32_t row = stg0 + buf * kEpiBufBytes;
 #pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
+          for (int cc = 0; cc < 2; ++cc) {
             uint32_t v[32];
-            tmem_ld32(taddr + h * kTile + cc * 32, v);
+            tmem_ld32(taddr + j * 64 + cc * 32, v);
             tmem_ld_wait();
-            if (h == BN / kTile - 1 && cc == 3) {
+            if (j == BN / 64 - 1 && cc == 1) {
               // last read of this accumulator: the MMA warp may overwrite it
               tc_fence_before();
               __syncwarp();
@@ -966,7 +1074,6 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
                 else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
               }
             }
-            const uint32_t box = stg + (cc >> 1) * 4096 + lane * 128;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               uint4 o;
@@ -977,34 +1084,88 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
                                                           __uint_as_float(v[8 * e + 2 * u + 1]));
                 ow[u] = *reinterpret_cast<uint32_t*>(&hh);
               }
-              const int chunk = (cc & 1) * 4 + e;  // 16-byte chunk inside the 128-byte row
-              st_shared_v4(box + ((chunk ^ (lane & 7)) << 4), o);
+              const int chunk = cc * 4 + e;  // 16-byte chunk inside the 128-byte row
+              st_shared_v4(row + ((chunk ^ (lane & 7)) << 4), o);
             }
           }
-          fence_async_smem();
+          fence_async_smem();  // the TMA store reads what this warp wrote
           __syncwarp();
-          if (lane == 0) {
-            const int x0 = nb * BN + h * kTile, y0 = mb * kBM + q * 32;
-            tma_store_2d(&maps.c_st, x0, y0, stg);
-            tma_store_2d(&maps.c_st, x0 + 64, y0, stg + 4096);
-            bulk_commit();
-            if (h == BN / kTile - 1) bulk_wait_done<0>();  // stores complete: publishable
-            else bulk_wait_read<0>();                      // staging may be rewritten
-          }
-          __syncwarp();
-        }
-        // all of the block's stores (of all four warps), then the flags (Sec. 4.2)
-        named_bar_sync(1, kEpiThreads);
-        if (warp == kEpiWarp0 && lane == 0) {
-          for (int c = 0; c < P.cpb; ++c) {
-            const int t = trow * P.nTn + nb * P.cpb + c;
-            st_release_gpu(&P.flags_own[d * P.Q + t], P.epoch);
-          }
-          published += P.cpb;
+          if (lane == 0) mbar_arrive(staged_bar(buf));
         }
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
       if (!ok && lane == 0) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -3); }
+    } else if (warp == kCStoreWarp && lane == 0) {
+      // ---- store thread: sends each staged box of the partial C with TMA, returns the staging
+      //      buffers, and counts the blocks whose stores are complete for the flag thread ----
+      int nbox = 0, freed = 0;  // boxes stored / boxes whose staging buffer has been returned
+      int n_issued = 0;         // blocks whose stores are all issued
+      int n_done = 0;           // blocks whose stores are known complete
+      bool ok = true;
+      auto free_upto = [&](int m) {
+        for (; freed <= m; ++freed) mbar_arrive(sfree_bar(freed & 1));
+      };
+      auto mark_done = [&](int n) {
+        if (n == n_done) return;
+        n_done = n;
+        st_release_cta(&sh.blocks_stored, n);
+      };
+      for (int i = 0; ok && i < n_my; ++i) {
+        int d, l;
+        block_of(i, &d, &l);
+        const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
+        for (int j = 0; j < BN / 64; ++j, ++nbox) {
+          const int buf = nbox & 1;
+          if (n_done < n_issued && !mbar_try_wait(staged_bar(buf), (nbox >> 1) & 1)) {
+            // the next box is not staged yet: time to see the issued stores complete
+            bulk_wait_done<0>();
+            free_upto(nbox - 1);
+            mark_done(n_issued);
+          }
+          if (!mbar_wait(staged_bar(buf), (nbox >> 1) & 1, P, &sh)) { ok = false; break; }
+          tma_store_2d(&maps.c_st, nb * BN + j * 64, mb * kBM,
+                       smem_base + n_stages * C::kStageBytes + buf * kEpiBufBytes);
+          bulk_commit();
+          bulk_wait_read<1>();  // the stores before this one have read their buffers
+          free_upto(nbox - 1);
+          if (n_done < n_issued) {
+            bulk_wait_done<1>();  // all stores but the one just issued, i.e. the earlier blocks'
+            mark_done(n_issued);
+          }
+        }
+        n_issued = i + 1;
+      }
+      bulk_wait_done<0>();
+      if (ok) mark_done(n_issued);
+      else { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -5); }
+    } else if (warp == kFlagWarp && lane == 0) {
+      // ---- flag thread: releases the tile flags of every block whose stores are complete
+      //      (Sec. 4.2).  The release fence takes about a microsecond when memory is busy; in a
+      //      thread of its own it delays neither the epilogue nor the stores ----
+      int seen = 0;
+      unsigned long long t0 = 0;
+      for (int i = 0; i < n_my; ++i) {
+        for (uint32_t spins = 1; seen <= i; ++spins) {
+          seen = ld_acquire_cta(&sh.blocks_stored);
+          if (seen > i) break;
+          __nanosleep(64);
+          if ((spins % kSpinCheck) == 0) {
+            if (sh.abort || global_abort(P)) break;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 64ULL * P.wait_budget_ns) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -6); break; }
+          }
+        }
+        if (seen <= i) break;
+        t0 = 0;
+        int d, l;
+        block_of(i, &d, &l);
+        const int t_first = (l / P.nBn) * P.nTn + (l % P.nBn) * P.cpb;
+        fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
+        fence_acq_rel_gpu();  // the stores seen complete by the store thread, then the flags
+        for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[d * P.Q + t_first + c], P.epoch);
+        published += P.cpb;
+      }
     }
     // ---- end of this CTA's producer work ----
     named_bar_sync(3, kGemmThreads);
@@ -1031,7 +1192,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       __threadfence_block();
       sh.gemm_done = 1;  // the consumer warps may take over the producer's shared memory
     }
-    if (warp == kEpiWarp0 && lane == 0 && published)
+    if (warp == kFlagWarp && lane == 0 && published)
       atomicAdd(&st->flags_published, (unsigned long long)published);
   } else if (comm_warp && P.mode != MODE_GEMM_ONLY) {
     // ---------------- consumer ----------------
@@ -1163,6 +1324,14 @@ static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS;
 }
+
+// Tasks per claim: as many as have their flags (W per reduce task) in the 64 flag values the
+// claiming warp reads ahead, at most two.  Longer claims measured slower where several CTAs
+// share a list: the tiles in flight at one time then lie further apart in memory.
+#ifndef ENTWINE_CLAIM_MAX
+#define ENTWINE_CLAIM_MAX 2
+#endif
+static int claim_size(int W) { return std::max(1, std::min(ENTWINE_CLAIM_MAX, 64 / W)); }
 
 int device_sm_count() {
   int n = 0;
@@ -1386,6 +1555,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.mode = mode;
   kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = (mode == MODE_COMM_ONLY) ? 1 : 0;
+  kp.claim = claim_size(g.W);
   kp.epoch = d->epoch;
   d->seq += 1;
   kp.seq = d->seq;
@@ -1441,7 +1611,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
                      kBK, kBM, true) &&
             make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
                      kBK, (mode != MODE_COMM_ONLY) ? (pair ? 128 : g.BN) : kBM, true) &&
-            make_map(&maps.c_st, d->C, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.c_st, d->C, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
@@ -1664,6 +1834,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.mode = MODE_FUSED;
   kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = 0;
+  kp.claim = claim_size(g.W);
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
@@ -1695,7 +1866,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   std::memset(&maps, 0, sizeof(maps));
   bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
             make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
-            make_map(&maps.c_st, base, g.M, g.N, 64, 32, true) &&
+            make_map(&maps.c_st, base, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];

@@ -20,7 +20,7 @@ if torch.cuda.is_available():
 FULL = [
     (I.ATTN_OUT, 1, (1, 0), (0, 20)),
     (I.MLP_DOWN, 5, (1,), (0, 20)),
-    (I.SHORT_K, 2, (1, 0), (8, 16, 24)),
+    (I.SHORT_K, 2, (1, 0), (0, 8, 16, 24)),
 ]
 
 
@@ -109,3 +109,34 @@ def test_sweep_corner_shapes_smoke_parity():
                 acc = acc + P[q, r * R:(r + 1) * R].float()
             assert torch.equal(out, acc.to(torch.bfloat16))
             p.destroy()
+
+
+def test_ring_handover_keeps_every_element_exact():
+    """Co-located consumers move from the small ring beside the producer's buffers to the large
+    ring that reuses those buffers when their CTA's producer work ends.  Steps still in flight
+    in the small ring at that moment must not be overwritten: with the communication-heavy
+    short-K shape (the consumers are busiest at the hand-over) and a poisoned workspace, every
+    pushed tile equals the stored partial bit for bit and every reduced element is the
+    rank-order fp32 sum, on repeated launches."""
+    wl, r = I.SHORT_K, 2
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    R, W = wl.R, wl.W
+    for order in (1, 0):
+        p = E.Plan(wl.M, wl.N, wl.K, W, order, 0, rank=r, poison_partial=1)
+        out = torch.empty((R, wl.N), dtype=torch.bfloat16, device="cuda")
+        send = torch.empty((W - 1, R, wl.N), dtype=torch.bfloat16, device="cuda")
+        Cd = torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device="cuda")
+        for _ in range(6):
+            out.fill_(float("nan"))
+            send.fill_(float("nan"))
+            p.gemm_rs(A, Bm, P, out, send)
+            p.read_partial(Cd)
+            torch.cuda.synchronize()
+            for slot, d in enumerate(dd for dd in range(W) if dd != r):
+                assert torch.equal(send[slot].view(torch.int16), Cd[d * R:(d + 1) * R].view(torch.int16))
+            acc = Cd[r * R:(r + 1) * R].float()
+            for q in range(W - 1):
+                acc = acc + P[q, r * R:(r + 1) * R].float()
+            assert torch.equal(out, acc.to(torch.bfloat16))
+        p.destroy()
