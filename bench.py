@@ -237,6 +237,18 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     res["status"] = st
     res["fused_hot_us"] = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), steps, 3, flush, torch, cold=False)
     plan.last_status()
+    # Back to back: `steps` calls queued between ONE event pair, no flush.  The queue hides the
+    # launch latency of all calls but the first; a call's streamed data (partial C, incoming
+    # partials, outputs) exceeds L2 for every configuration but the tiny one, so L2 holds at
+    # most the operands when the next call starts.
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        plan.gemm_rs(A, Bm, P, out, send)
+    e1.record()
+    torch.cuda.synchronize()
+    res["fused_back_to_back_us"] = e0.elapsed_time(e1) * 1e3 / steps
+    plan.last_status()
     if detailed:
         # the producer alone (uncontended GEMM time) and the consumer alone
         res["gemm_only_us"] = time_steps(lambda: plan.gemm_only(A, Bm), max(5, steps // 4), 3, flush, torch)
@@ -511,6 +523,7 @@ def main():
             e = {
                 "fused_us": fused, "fused_tflops": w2.flops / fused / 1e6,
                 "fused_hot_l2_us": med(r["fused_hot_us"]),
+                "fused_back_to_back_us": r["fused_back_to_back_us"],
                 "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
                 "bound": "tensor" if tc >= hb else "hbm",
                 "unfused_cublas_then_reduce_us": med(r["unfused_us"]),

@@ -59,6 +59,9 @@ enum {
   ENTWINE_ERR_TOO_LARGE = -6  /* the problem does not fit entwine_gemm_rs_static's fixed scratch */
 };
 
+/* Values of ENTWINE_OPT_RELEASE_GROUP besides a block count. */
+enum { ENTWINE_RELEASE_PARTITION = -1, ENTWINE_RELEASE_WHOLE = -2 };
+
 /* Option keys for entwine_set_option. Options marked [pre] must be set before the first
  * launch of the plan; the others may change between launches. */
 enum {
@@ -91,6 +94,14 @@ enum {
                                       own partition goes to list t mod x); 0 (default): one list
                                       per consumer CTA.  With fewer lists than CTAs the CTAs share
                                       lists through the lists' head counters                     */
+  ENTWINE_OPT_RELEASE_GROUP   = 14, /* release granularity of the tile flags (the ablation of Sec. 5,
+                                      "Release Granularity"; each reduction task stays one tile):
+                                      1 (default): a producer block's tiles are released when the
+                                      block is stored; g > 1: g consecutive blocks of the tile order
+                                      are released together, when the last of them is stored;
+                                      ENTWINE_RELEASE_PARTITION (-1): all tiles of a destination
+                                      partition together; ENTWINE_RELEASE_WHOLE (-2): the whole
+                                      output together.  Results are identical for every value      */
   ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */

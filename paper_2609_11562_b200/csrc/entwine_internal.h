@@ -77,6 +77,7 @@ struct Plan {
   int prefetch = 0;         // look-ahead L2 prefetch of peer tiles (measured: no gain)
   int l2_hints = 3;         // bit 0: evict-first on the consumer's TMA traffic, bit 1: evict-last on operands
   int lists_opt = 0;        // number of consumer lists x, 0 = one per consumer CTA
+  int release_group = 1;    // blocks released together; -1 per destination partition, -2 whole output
   int stages = 0;           // operand-ring stages of the producer, 0 = choose
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles

@@ -95,6 +95,8 @@ struct KParams {
   int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
   int skip_wait;  // treat every flag as published (consumer in isolation)
   int claim;      // most consecutive tasks taken from a list per claim
+  int release_group;     // blocks released together (1 = each block by itself; -1, -2: see the header)
+  unsigned* group_ctr;   // stored blocks per release group (counts modulo the group's size)
   // consumer ring geometry, [0] ring A (small, beside the producer's buffers), [1] ring B
   int rs[2];         // rows of a tile moved per reduce step (all W contributions of those rows)
   int prs[2];        // rows of a tile moved per push step
@@ -964,11 +966,14 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     // ---------------- producer: tcgen05 GEMM ----------------
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(smem + kBarOff + kBarTmemSlot);
     const int KB = (P.K + kBK - 1) / kBK;
+    // block i of this CTA: its position in the tile order (returned), its destination partition
+    // d and its index l inside the partition
     auto block_of = [&](int i, int* d, int* l) {
       const int unit = unit0 + i * stride;
       const int p = PAIR ? pair_position(P, unit, (int)cta_rank) : unit;
       if (P.order == ENTWINE_ORDER_INTERLEAVED) { *d = p % P.W; *l = p / P.W; }
       else { *d = p / P.Lb; *l = p - *d * P.Lb; }
+      return p;
     };
 
     if (warp == kTmaWarp && lane == 0) {
@@ -1159,12 +1164,40 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         if (seen <= i) break;
         t0 = 0;
         int d, l;
-        block_of(i, &d, &l);
-        const int t_first = (l / P.nBn) * P.nTn + (l % P.nBn) * P.cpb;
+        const int pos = block_of(i, &d, &l);
+        auto release_block = [&](int dd, int ll) {
+          const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb;
+          for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
+          published += P.cpb;
+        };
         fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
         fence_acq_rel_gpu();  // the stores seen complete by the store thread, then the flags
-        for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[d * P.Q + t_first + c], P.epoch);
-        published += P.cpb;
+        if (P.release_group == 1) {
+          release_block(d, l);
+          continue;
+        }
+        // Coarser release (the granularity ablation): the block is counted in its group; whoever
+        // stores a group's last block releases the flags of all its blocks.  The counter is never
+        // reset: every launch adds the group's size to it.
+        int gid, gsize, first = 0;
+        if (P.release_group == ENTWINE_RELEASE_WHOLE) { gid = 0; gsize = P.P_blk; }
+        else if (P.release_group == ENTWINE_RELEASE_PARTITION) { gid = d; gsize = P.Lb; }
+        else {
+          gid = pos / P.release_group;
+          first = gid * P.release_group;
+          gsize = min(P.release_group, P.P_blk - first);
+        }
+        const unsigned prev = atomicAdd(&P.group_ctr[gid], 1u);
+        if ((prev + 1u) % (unsigned)gsize != 0u) continue;
+        fence_acq_rel_gpu();  // the other blocks' stores, released by their CTAs' counts
+        if (P.release_group == ENTWINE_RELEASE_PARTITION) {
+          for (int ll = 0; ll < P.Lb; ++ll) release_block(d, ll);
+        } else {
+          for (int pp = first; pp < first + gsize; ++pp) {
+            if (P.order == ENTWINE_ORDER_INTERLEAVED) release_block(pp % P.W, pp / P.W);
+            else release_block(pp / P.Lb, pp % P.Lb);
+          }
+        }
       }
     }
     // ---- end of this CTA's producer work ----
@@ -1265,6 +1298,7 @@ struct DeviceState {
   int* list_head = nullptr;
   StatusSlot* status = nullptr;
   unsigned* done_ctr = nullptr;
+  unsigned* group_ctr = nullptr;
   unsigned epoch = 0;
   unsigned seq = 0;
   bool status_pending = false;
@@ -1376,7 +1410,8 @@ static int ensure_device(Plan* p) {
             cudaMalloc(&d->list_offs, t.list_offs.size() * 4) == cudaSuccess &&
             cudaMalloc(&d->list_head, size_t(p->x) * 4) == cudaSuccess &&
             cudaMalloc(&d->status, 2 * sizeof(StatusSlot)) == cudaSuccess &&
-            cudaMalloc(&d->done_ctr, 4) == cudaSuccess;
+            cudaMalloc(&d->done_ctr, 4) == cudaSuccess &&
+            cudaMalloc(&d->group_ctr, size_t(g.P_blk) * 4) == cudaSuccess;
   if (ok) {
     StatusSlot init[2];
     std::memset(init, 0, sizeof(init));
@@ -1390,7 +1425,8 @@ static int ensure_device(Plan* p) {
              cudaSuccess &&
          cudaMemset(d->list_head, 0, size_t(p->x) * 4) == cudaSuccess &&
          cudaMemcpy(d->status, init, sizeof(init), cudaMemcpyHostToDevice) == cudaSuccess &&
-         cudaMemset(d->done_ctr, 0, 4) == cudaSuccess;
+         cudaMemset(d->done_ctr, 0, 4) == cudaSuccess &&
+         cudaMemset(d->group_ctr, 0, size_t(g.P_blk) * 4) == cudaSuccess;
   }
   p->dev = d;
   if (!ok) {
@@ -1417,6 +1453,7 @@ void device_release(Plan* p) {
   cudaFree(d->list_head);
   cudaFree(d->status);
   cudaFree(d->done_ctr);
+  cudaFree(d->group_ctr);
   cudaFree(d->sA);
   cudaFree(d->sB);
   cudaFree(d->sPeers);
@@ -1530,6 +1567,8 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
       d->epoch = 1;
     }
     if (p->poison) CK(cudaMemsetAsync(d->C, 0xff, size_t(g.M) * g.N * 2, stream));
+    // coarse release only: start the group counts from zero whatever an earlier launch left
+    if (p->release_group != 1) CK(cudaMemsetAsync(d->group_ctr, 0, size_t(g.P_blk) * 4, stream));
   }
   if (d->withheld != p->withhold_peer) {
     // host-side fault injection: a peer flag that is never published
@@ -1555,6 +1594,8 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.mode = mode;
   kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = (mode == MODE_COMM_ONLY) ? 1 : 0;
+  kp.release_group = p->release_group;
+  kp.group_ctr = d->group_ctr;
   kp.claim = claim_size(g.W);
   kp.epoch = d->epoch;
   d->seq += 1;
@@ -1834,6 +1875,8 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.mode = MODE_FUSED;
   kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;  // shared lists need every CTA to scan them
   kp.skip_wait = 0;
+  kp.release_group = 1;  // this entry point keeps the per-block release
+  kp.group_ctr = nullptr;
   kp.claim = claim_size(g.W);
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;

@@ -257,6 +257,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       if (p->launched || value < 0 || value > 4096) return ENTWINE_ERR_INVALID;
       p->lists_opt = int(value);
       return entwine::finalize_plan(p);
+    case ENTWINE_OPT_RELEASE_GROUP:
+      if (value == 0 || value < ENTWINE_RELEASE_WHOLE || value > (int64_t(1) << 24)) return ENTWINE_ERR_INVALID;
+      p->release_group = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_STAGES:
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);

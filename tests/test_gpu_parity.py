@@ -292,6 +292,9 @@ def test_host_buffer_entry_point():
 OPTION_SETS = [
     dict(colocate=0), dict(colocate=0, tail_help=0), dict(stages=3), dict(stages=4), dict(stages=5),
     dict(prefetch=1), dict(pair_ctas=0, stages=3), dict(tail_help=0), dict(l2_hints=0), dict(l2_hints=1), dict(lists=1), dict(lists=5),
+    # release granularity (Sec. 5 ablation): groups of blocks, a partition, the whole output
+    dict(release_group=3), dict(release_group=16), dict(release_group=-1), dict(release_group=-2),
+    dict(release_group=5, pair_ctas=0), dict(release_group=-1, colocate=0, tail_help=0),
 ]
 
 

@@ -140,3 +140,17 @@ def test_launch_without_device_fails_loudly():
         p.gemm_rs(16, 16, 16, 16, 16, stream=0)
     assert e.value.code == E.ERR_CUDA
     p.destroy()
+
+
+def test_release_group_option_validation():
+    """ENTWINE_OPT_RELEASE_GROUP accepts a block count >= 1, the partition and whole-output
+    values, and nothing else; it leaves the plan's tables untouched."""
+    p = E.Plan(1024, 1024, 256, 4, 1, 4, num_sms=148)
+    before = p.export(E.EXPORT_TASKS).copy()
+    for ok in (1, 2, 7, 1000, E.RELEASE_PARTITION, E.RELEASE_WHOLE):
+        p.set_option(E.OPT_RELEASE_GROUP, ok)
+    for bad in (0, -3, 1 << 25):
+        with pytest.raises(E.EntwineError):
+            p.set_option(E.OPT_RELEASE_GROUP, bad)
+    assert np.array_equal(before, p.export(E.EXPORT_TASKS))
+    p.destroy()
