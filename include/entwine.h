@@ -46,7 +46,10 @@ typedef struct entwine_plan_s* entwine_plan_t;
 /* Producer tile orders (Sec. 3.1 and Fig. 1). */
 enum {
   ENTWINE_ORDER_ROW_MAJOR   = 0, /* partition-grouped: all blocks of partition 0, then 1, ... */
-  ENTWINE_ORDER_INTERLEAVED = 1  /* Eq. 1: d = p mod W, l = floor(p / W)                      */
+  ENTWINE_ORDER_INTERLEAVED = 1, /* Eq. 1: d = p mod W, l = floor(p / W)                      */
+  ENTWINE_ORDER_M_MAJOR     = 2  /* ablation baseline (Sec. 5, "Computation Order"): the block
+                                    grid of the whole output walked down the rows first, one
+                                    block column after another, regardless of partitions      */
 };
 
 enum {

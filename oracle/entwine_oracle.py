@@ -43,6 +43,7 @@ T = 128  # reduction-tile edge (Sec. 4.2)
 
 ORDER_ROW_MAJOR = 0    # partition-grouped traversal (Fig. 1, top)
 ORDER_INTERLEAVED = 1  # Eq. 1 (Fig. 1, bottom)
+ORDER_M_MAJOR = 2      # the producer kernel's default traversal in the order ablation (Sec. 5.3.1)
 
 KIND_REDUCE = 0
 KIND_PUSH = 1
@@ -98,6 +99,9 @@ def schedule(M: int, N: int, W: int, BN: int, order: int):
     Interleaved order is Eq. 1: d = p mod W, l = floor(p / W).
     Row-major order is the partition-grouped traversal of Fig. 1 (top): all blocks of
     partition 0, then partition 1, ...
+    M-major order is the baseline of the computation-order ablation (Sec. 5.3.1): the block
+    grid of the whole output is walked down the rows first, one block column after another,
+    ignoring partitions and the consumer's order.
     Inside a partition l walks the block grid with the column index fastest (the
     "N-major" consumer order of Sec. 5.3.1), and tiles are numbered row-major over the
     partition's 128 x 128 grid, so a 128 x 256 block covers two consecutive tile indices
@@ -116,6 +120,13 @@ def schedule(M: int, N: int, W: int, BN: int, order: int):
         elif order == ORDER_ROW_MAJOR:
             dp = p // g.Lb
             lp = p % g.Lb
+        elif order == ORDER_M_MAJOR:
+            # the block grid of the whole M x N output walked with the row index fastest
+            rows_all = W * g.rowsT           # block rows of the output
+            row_all = p % rows_all
+            col_all = p // rows_all
+            dp = row_all // g.rowsT
+            lp = (row_all % g.rowsT) * g.nBn + col_all
         else:
             raise ValueError("unknown tile order")
         row_in_part = lp // g.nBn   # tile row inside the partition

@@ -397,8 +397,25 @@ __device__ __forceinline__ constexpr uint32_t instr_desc() {
 // a pair share the block column (the B panel).  Interleaved order (W even): positions 2u and
 // 2u+1 of Eq. 1, i.e. two destinations at once.  Row-major order (even tile rows per
 // partition): vertically adjacent blocks of one partition.
+// Destination partition d and block index l inside the partition of position p of the tile
+// order (Eq. 1 for the interleaved order).
+__device__ __forceinline__ void position_to_block(const KParams& P, int p, int* d, int* l) {
+  if (P.order == ENTWINE_ORDER_INTERLEAVED) {
+    *d = p % P.W;
+    *l = p / P.W;
+  } else if (P.order == ENTWINE_ORDER_M_MAJOR) {
+    const int rows_all = P.W * P.rowsT;
+    const int row_all = p % rows_all, col_all = p / rows_all;
+    *d = row_all / P.rowsT;
+    *l = (row_all - *d * P.rowsT) * P.nBn + col_all;
+  } else {
+    *d = p / P.Lb;
+    *l = p - *d * P.Lb;
+  }
+}
 __device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) {
-  if (P.order == ENTWINE_ORDER_INTERLEAVED) return 2 * u + rank;
+  // interleaved and M-major: consecutive positions share a block column
+  if (P.order != ENTWINE_ORDER_ROW_MAJOR) return 2 * u + rank;
   const int half = P.Lb / 2;
   const int d = u / half, rem = u - d * half;
   const int v = rem / P.nBn, nb = rem - v * P.nBn;
@@ -971,8 +988,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     auto block_of = [&](int i, int* d, int* l) {
       const int unit = unit0 + i * stride;
       const int p = PAIR ? pair_position(P, unit, (int)cta_rank) : unit;
-      if (P.order == ENTWINE_ORDER_INTERLEAVED) { *d = p % P.W; *l = p / P.W; }
-      else { *d = p / P.Lb; *l = p - *d * P.Lb; }
+      position_to_block(P, p, d, l);
       return p;
     };
 
@@ -1194,8 +1210,9 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           for (int ll = 0; ll < P.Lb; ++ll) release_block(d, ll);
         } else {
           for (int pp = first; pp < first + gsize; ++pp) {
-            if (P.order == ENTWINE_ORDER_INTERLEAVED) release_block(pp % P.W, pp / P.W);
-            else release_block(pp / P.Lb, pp % P.Lb);
+            int dd, ll;
+            position_to_block(P, pp, &dd, &ll);
+            release_block(dd, ll);
           }
         }
       }

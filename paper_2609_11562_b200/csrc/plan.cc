@@ -37,6 +37,11 @@ void block_of_position(const Geometry& g, int order, int p, int* mb, int* nb, in
   if (order == ENTWINE_ORDER_INTERLEAVED) {  // Eq. 1
     dest = p % g.W;
     ell = p / g.W;
+  } else if (order == ENTWINE_ORDER_M_MAJOR) {  // rows of the whole output first
+    const int rows_all = g.W * g.rowsT;
+    const int row_all = p % rows_all, col_all = p / rows_all;
+    dest = row_all / g.rowsT;
+    ell = (row_all - dest * g.rowsT) * g.nBn + col_all;
   } else {  // partition-grouped traversal (Fig. 1, top)
     dest = p / g.Lb;
     ell = p - dest * g.Lb;
@@ -152,7 +157,8 @@ int finalize_plan(Plan* p) {
   const Geometry& g = p->g;
   p->pair = p->pair_opt && g.BN == 256 && p->num_sms >= 2 &&
             ((p->order == ENTWINE_ORDER_INTERLEAVED && g.W % 2 == 0) ||
-             (p->order == ENTWINE_ORDER_ROW_MAJOR && g.rowsT % 2 == 0));
+             (p->order == ENTWINE_ORDER_ROW_MAJOR && g.rowsT % 2 == 0) ||
+             (p->order == ENTWINE_ORDER_M_MAJOR && (g.W * g.rowsT) % 2 == 0));
   if (p->n_comm_sms == 0) {
     // non-overlapped use of all SMs: every CTA produces, then consumes
     p->n_comm_ctas = 0;
@@ -181,7 +187,8 @@ int entwine_plan(entwine_plan_t* plan, int64_t M, int64_t N, int64_t K_local, in
                  int tile_order, int n_comm_sms) {
   if (!plan) return ENTWINE_ERR_INVALID;
   *plan = nullptr;
-  if (tile_order != ENTWINE_ORDER_ROW_MAJOR && tile_order != ENTWINE_ORDER_INTERLEAVED)
+  if (tile_order != ENTWINE_ORDER_ROW_MAJOR && tile_order != ENTWINE_ORDER_INTERLEAVED &&
+      tile_order != ENTWINE_ORDER_M_MAJOR)
     return ENTWINE_ERR_INVALID;
   entwine::Geometry g;
   if (!entwine::make_geometry(M, N, K_local, W, 256, &g)) {

@@ -20,7 +20,7 @@ if not os.path.exists(LIB_PATH):
         "(or __graft_entry__.build()); this package has no CPU fallback")
 _lib = ctypes.CDLL(LIB_PATH)
 
-ORDER_ROW_MAJOR, ORDER_INTERLEAVED = 0, 1
+ORDER_ROW_MAJOR, ORDER_INTERLEAVED, ORDER_M_MAJOR = 0, 1, 2
 OK, ERR_INVALID, ERR_RESOURCES, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2, -3, -4, -5
 ERR_TOO_LARGE = -6
 OPT_RANK, OPT_BLOCK_N, OPT_WAIT_BUDGET_NS, OPT_TAIL_HELP = 1, 2, 3, 4

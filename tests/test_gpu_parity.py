@@ -193,6 +193,40 @@ def test_fused_matches_oracle(wl):
             p.destroy()
 
 
+@pytest.mark.parametrize("wl", [SMALL[1], SMALL[4]], ids=lambda w: w.name)
+def test_m_major_order_matches_oracle_and_the_other_orders(wl):
+    """The ablation's baseline order (Sec. 5.3.1) changes when tiles appear, not what is
+    computed: oracle tolerance, exact counts, and results bit-identical to Eq. 1's order."""
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    Ad, Bd, Pd = A.cuda(), Bm.cuda(), P.cuda()
+    r = wl.W - 1
+    ref_plan = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r)
+    out0, send0 = _alloc_outputs(wl)
+    ref_plan.gemm_rs(Ad, Bd, Pd, out0, send0)
+    ref_plan.last_status()
+    ref_plan.destroy()
+    for BN, n_comm, pair, rel in itertools.product((128, 256), (0, 4, 20), (0, 1), (1, 4)):
+        if wl.N % BN or (pair and BN == 128):
+            continue
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_M_MAJOR, n_comm, block_n=BN, rank=r, pair_ctas=pair,
+                   release_group=rel)
+        c = p.counts()
+        res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, BN, O.ORDER_M_MAJOR, c["x"])
+        out, send = _alloc_outputs(wl)
+        p.gemm_rs(Ad, Bd, Pd, out, send)
+        st = p.last_status()
+        assert st["flags_published"] == c["flags_published"] == wl.W * c["Q"]
+        assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+        if _tolerance_is_feasible(wl):
+            _check_against_oracle(wl, r, res, out, send)
+        else:
+            _check_against_staged(wl, r, res, Ab, Bb, Pb, out, send)
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        p.destroy()
+
+
 def test_fused_is_deterministic_and_ordered_under_poison():
     """Single writer per element (Sec. 4.2) => bitwise reproducible; with the partial-output
     workspace refilled with NaN patterns before each call, any read that overtakes the

@@ -69,7 +69,7 @@ CASES = [(256, 256, 128, 2), (512, 768, 64, 4), (384, 384, 64, 3), (2048, 1280, 
 @pytest.mark.parametrize("M,N,K,W", CASES)
 def test_exported_tables_equal_oracle(M, N, K, W):
     big = M * N > 2 ** 22
-    orders = (E.ORDER_ROW_MAJOR, E.ORDER_INTERLEAVED)
+    orders = (E.ORDER_ROW_MAJOR, E.ORDER_INTERLEAVED, E.ORDER_M_MAJOR)
     bns = [bn for bn in (128, 256) if N % bn == 0]
     ranks = (W - 1,) if big else (0, W - 1)
     budgets = (20,) if big else (0, 1, 4, 24)
@@ -81,7 +81,8 @@ def test_exported_tables_equal_oracle(M, N, K, W):
         # CTA-pair tiles (two blocks sharing a block column) need an even number of producers
         rowsT = M // W // 128
         pair = BN == 256 and ((order == E.ORDER_INTERLEAVED and W % 2 == 0) or
-                              (order == E.ORDER_ROW_MAJOR and rowsT % 2 == 0))
+                              (order == E.ORDER_ROW_MAJOR and rowsT % 2 == 0) or
+                              (order == E.ORDER_M_MAJOR and (W * rowsT) % 2 == 0))
         want_g = (148 - n_comm) & ~1 if pair else 148 - n_comm
         assert c["n_gemm_ctas"] == want_g and c["n_comm_ctas"] == n_comm
         s = O.schedule(M, N, W, BN, order)

@@ -116,6 +116,35 @@ def test_eq1_closed_form_and_bijection(M, N, W, BN):
         assert _longest_local_run(b["d"], r) == 1
 
 
+@pytest.mark.parametrize("M,N,W", SHAPES)
+@pytest.mark.parametrize("BN", [128, 256])
+def test_m_major_order_is_column_major_walk_of_the_block_grid(M, N, W, BN):
+    """The ablation's baseline order (Sec. 5.3.1) written out as a brute-force enumeration:
+    for every block column, every block row of the whole output from top to bottom."""
+    if N % BN:
+        pytest.skip("N not a multiple of BN")
+    s = O.schedule(M, N, W, BN, O.ORDER_M_MAJOR)
+    g = s["geom"]
+    walk = [(row, col) for col in range(N // BN) for row in range(M // 128)]
+    assert list(zip(s["mb"].tolist(), s["nb"].tolist())) == walk
+    assert O.check_every_tile_once(s)
+    assert (s["mb"] // g.rowsT == s["d"]).all()
+    assert (s["l"] == (s["mb"] - s["d"] * g.rowsT) * g.nBn + s["nb"]).all()
+    for pp in range(g.P_blk):
+        for c in range(g.cpb):
+            t = s["tiles"][pp, c]
+            assert t // g.nTn == s["mb"][pp] - s["d"][pp] * g.rowsT
+            assert t % g.nTn == s["nb"][pp] * g.cpb + c
+    # same set of blocks as Eq. 1; consecutive local blocks come in runs of one partition's
+    # block rows (rowsT), not Lb and not 1
+    b = O.schedule(M, N, W, BN, O.ORDER_INTERLEAVED)
+    assert sorted(zip(s["mb"], s["nb"])) == sorted(zip(b["mb"], b["nb"]))
+    for r in range(W):
+        # rank W-1's run at the bottom of one column is not followed by its own blocks; the
+        # others likewise: every run is exactly one partition's rows of one block column
+        assert _longest_local_run(s["d"], r) == g.rowsT
+
+
 def test_tile_numbering_same_for_both_block_widths():
     # the consumer uses the same 128x128 tiles with either producer (Sec. 4.2)
     for order in (0, 1):
