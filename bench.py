@@ -316,6 +316,64 @@ def run_sweep(args, peaks, flush, torch, E, I):
     return 0
 
 
+def run_ablation(args, peaks, flush, torch, E, I):
+    """The design ablations of Sec. 5 on this GPU: computation order, release granularity and
+    SM sharing, each on a short-K and a long-K shape.  Every variant is the same kernel with
+    another plan option; each line reports the variant's best communication budget."""
+    iters = args.sweep_iters
+    shapes = [I.Workload("ablation_short_K", 8, 8192, 8192, 1024, "normal_fanin", "normal_fanin", 6, 0),
+              I.Workload("ablation_long_K", 8, 8192, 8192, 4096, "normal_fanin", "normal_fanin", 6, 1)]
+    report = {}
+    for wl in shapes:
+        A, Bm = I.make_operands(wl, device="cuda")
+        P = I.make_peer_partials(wl, device="cuda")
+        out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+
+        def fused(order, n_comm, **opts):
+            plan = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=wl.W - 1, **opts)
+            us = statistics.median(time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), iters, 3, flush, torch))
+            st = plan.last_status()
+            plan.destroy()
+            return {"fused_us": us, "t_gemm_us": st["t_gemm_ns"] / 1e3,
+                    "tail_us": (st["t_end_ns"] - st["t_gemm_ns"]) / 1e3, "n_comm_sms": n_comm}
+
+        def best(order, budgets, **opts):
+            return min((fused(order, b, **opts) for b in budgets), key=lambda r: r["fused_us"])
+
+        plan = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=wl.W - 1)
+        gemm_us = statistics.median(time_steps(lambda: plan.gemm_only(A, Bm), iters, 3, flush, torch))
+        plan.last_status()
+        comm_us = statistics.median(time_steps(lambda: plan.comm_only(None, P, out, send, 0), iters, 3, flush, torch))
+        plan.last_status()
+        plan.destroy()
+        base = gemm_us + comm_us  # the non-overlapped baseline: producer alone, then consumer alone
+        budgets = (0, 8, 16, 32)
+        rec = {"shape": {"W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K},
+               "non_overlapped_us": base, "gemm_alone_us": gemm_us, "comm_alone_us": comm_us}
+        rec["computation_order"] = {name: best(order, budgets) for name, order in
+                                    (("interleaved", 1), ("row_major", 0), ("m_major", 2))}
+        gran = {}
+        for name, g in (("block", 1), ("4_blocks", 4), ("16_blocks", 16), ("64_blocks", 64),
+                        ("partition", E.RELEASE_PARTITION), ("whole_output", E.RELEASE_WHOLE)):
+            r = best(1, (0, 16), release_group=g)
+            r["speedup_vs_non_overlapped"] = base / r["fused_us"]
+            gran[name] = r
+        rec["release_granularity"] = gran
+        rec["sm_sharing"] = {
+            "shared_pool": best(1, budgets),
+            "static_partition": best(1, (8, 16, 24, 32, 48, 64), colocate=0, tail_help=0),
+        }
+        report[wl.name] = rec
+        del A, Bm, P, out, send
+        torch.cuda.empty_cache()
+    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+    with open(os.path.join(ROOT, "gpurun_out", "ablation.json"), "w") as f:
+        json.dump(report, f, indent=1)
+    print(json.dumps({"ablation": report}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -330,6 +388,9 @@ def main():
                          "JSON line per point to --sweep-out and print a summary line")
     ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
     ap.add_argument("--sweep-iters", type=int, default=8)
+    ap.add_argument("--ablation", action="store_true",
+                    help="the design ablations (computation order, release granularity, SM sharing) on a "
+                         "short-K and a long-K shape; prints one JSON line and writes gpurun_out/ablation.json")
     ap.add_argument("--comm-curve", action="store_true",
                     help="consumer bandwidth in isolation against the number of consumer CTAs (App. A)")
     ap.add_argument("--comm-ctas", type=int, default=0,
@@ -366,6 +427,8 @@ def main():
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB of L2
     if args.sweep:
         return run_sweep(args, peaks, flush, torch, E, I)
+    if args.ablation:
+        return run_ablation(args, peaks, flush, torch, E, I)
     if args.comm_curve:
         # every input available, no competing producer: bandwidth against the budget (App. A)
         A, Bm = I.make_operands(wl, device="cuda")

@@ -475,7 +475,7 @@ __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
       if (t0 == 0) t0 = now;
       else if (now - t0 > P.wait_budget_ns) return false;
     }
-    __nanosleep(64);
+    __nanosleep(64);  // longer, growing pauses (up to 4 us) were measured: no effect on the producer
   }
 }
 
@@ -1159,63 +1159,82 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       bulk_wait_done<0>();
       if (ok) mark_done(n_issued);
       else { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -5); }
-    } else if (warp == kFlagWarp && lane == 0) {
-      // ---- flag thread: releases the tile flags of every block whose stores are complete
+    } else if (warp == kFlagWarp) {
+      // ---- flag warp: releases the tile flags of every block whose stores are complete
       //      (Sec. 4.2).  The release fence takes about a microsecond when memory is busy; in a
-      //      thread of its own it delays neither the epilogue nor the stores ----
+      //      warp of its own it delays neither the epilogue nor the stores.  Lane 0 waits and
+      //      counts; a group release (the granularity ablation) is spread over the lanes ----
       int seen = 0;
       unsigned long long t0 = 0;
+      auto release_block = [&](int dd, int ll) {
+        const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb;
+        for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
+        published += P.cpb;
+      };
       for (int i = 0; i < n_my; ++i) {
-        for (uint32_t spins = 1; seen <= i; ++spins) {
-          seen = ld_acquire_cta(&sh.blocks_stored);
-          if (seen > i) break;
-          __nanosleep(64);
-          if ((spins % kSpinCheck) == 0) {
-            if (sh.abort || global_abort(P)) break;
-            const unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 64ULL * P.wait_budget_ns) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -6); break; }
-          }
-        }
-        if (seen <= i) break;
-        t0 = 0;
         int d, l;
         const int pos = block_of(i, &d, &l);
-        auto release_block = [&](int dd, int ll) {
-          const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb;
-          for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
-          published += P.cpb;
-        };
-        fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
-        fence_acq_rel_gpu();  // the stores seen complete by the store thread, then the flags
-        if (P.release_group == 1) {
-          release_block(d, l);
-          continue;
+        // what lane 0 finds: 0 = stop (abort / timeout), 1 = nothing to release for this block,
+        // 2 = release the group [first, first + gsize) (or partition d)
+        int verdict = 0, first = 0, gsize = 1;
+        if (lane == 0) {
+          for (uint32_t spins = 1; seen <= i; ++spins) {
+            seen = ld_acquire_cta(&sh.blocks_stored);
+            if (seen > i) break;
+            __nanosleep(64);
+            if ((spins % kSpinCheck) == 0) {
+              if (sh.abort || global_abort(P)) break;
+              const unsigned long long now = globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > 64ULL * P.wait_budget_ns) {
+                sh.abort = 1;
+                report(P, -ENTWINE_ERR_TIMEOUT, -6);
+                break;
+              }
+            }
+          }
+          if (seen > i) {
+            t0 = 0;
+            fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
+            fence_acq_rel_gpu();  // the stores seen complete by the store thread, then the flags
+            if (P.release_group == 1) {
+              release_block(d, l);
+              verdict = 1;
+            } else {
+              // Coarser release: the block is counted in its group; whoever stores a group's
+              // last block releases the flags of all its blocks.  Counts are taken modulo the
+              // group's size: every launch adds exactly that much.
+              int gid;
+              if (P.release_group == ENTWINE_RELEASE_WHOLE) { gid = 0; gsize = P.P_blk; }
+              else if (P.release_group == ENTWINE_RELEASE_PARTITION) { gid = d; gsize = P.Lb; }
+              else {
+                gid = pos / P.release_group;
+                first = gid * P.release_group;
+                gsize = min(P.release_group, P.P_blk - first);
+              }
+              const unsigned prev = atomicAdd(&P.group_ctr[gid], 1u);
+              verdict = ((prev + 1u) % (unsigned)gsize == 0u) ? 2 : 1;
+            }
+          }
         }
-        // Coarser release (the granularity ablation): the block is counted in its group; whoever
-        // stores a group's last block releases the flags of all its blocks.  The counter is never
-        // reset: every launch adds the group's size to it.
-        int gid, gsize, first = 0;
-        if (P.release_group == ENTWINE_RELEASE_WHOLE) { gid = 0; gsize = P.P_blk; }
-        else if (P.release_group == ENTWINE_RELEASE_PARTITION) { gid = d; gsize = P.Lb; }
-        else {
-          gid = pos / P.release_group;
-          first = gid * P.release_group;
-          gsize = min(P.release_group, P.P_blk - first);
-        }
-        const unsigned prev = atomicAdd(&P.group_ctr[gid], 1u);
-        if ((prev + 1u) % (unsigned)gsize != 0u) continue;
+        verdict = __shfl_sync(0xffffffffu, verdict, 0);
+        if (verdict == 0) break;
+        if (verdict == 1) continue;
+        first = __shfl_sync(0xffffffffu, first, 0);
+        gsize = __shfl_sync(0xffffffffu, gsize, 0);
         fence_acq_rel_gpu();  // the other blocks' stores, released by their CTAs' counts
-        if (P.release_group == ENTWINE_RELEASE_PARTITION) {
-          for (int ll = 0; ll < P.Lb; ++ll) release_block(d, ll);
-        } else {
-          for (int pp = first; pp < first + gsize; ++pp) {
+        for (int j = lane; j < gsize; j += 32) {
+          if (P.release_group == ENTWINE_RELEASE_PARTITION) {
+            release_block(d, j);
+          } else {
             int dd, ll;
-            position_to_block(P, pp, &dd, &ll);
+            position_to_block(P, first + j, &dd, &ll);
             release_block(dd, ll);
           }
         }
       }
+      // every lane's count of released flags, summed into lane 0
+      for (int o = 16; o > 0; o >>= 1) published += __shfl_down_sync(0xffffffffu, published, o);
     }
     // ---- end of this CTA's producer work ----
     named_bar_sync(3, kGemmThreads);
