@@ -40,9 +40,26 @@ NCU_TRAFFIC_BYTES = {"attn_out_proj": 55.41e6, "mlp_down_proj": 856.11e6, "short
 LAUNCH = {
     "attn_out_proj": dict(n_comm_sms=0, order=1, rank=1),
     "mlp_down_proj": dict(n_comm_sms=0, order=1, rank=5),
-    "short_k_comm_bound": dict(n_comm_sms=16, order=0, rank=2),
+    "short_k_comm_bound": dict(n_comm_sms=0, order=1, rank=2),
     "tiny": dict(n_comm_sms=4, order=1, rank=0),
 }
+
+
+def apply_tuned_table():
+    """Overlays the package's tuning table (written by paper_2609_11562_b200.autotune on a B200)
+    on LAUNCH: tile order, budget, and the producer options the tuner chose."""
+    from paper_2609_11562_b200 import autotune as T
+    from paper_2609_11562_b200 import inputs as I
+    path = os.path.join(ROOT, "paper_2609_11562_b200", "tuned_b200.json")
+    if not os.path.exists(path):
+        return
+    table = T.load_table(path)
+    for name, cfg in LAUNCH.items():
+        wl = I.CONFIGS[name]
+        if T.shape_key(wl.M, wl.N, wl.K, wl.W) not in table["shapes"]:
+            continue
+        order, n_comm, opts = T.launch_options(table, wl.M, wl.N, wl.K, wl.W)
+        cfg.update(order=order, n_comm_sms=n_comm, opts=opts)
 
 
 def load_peaks():
@@ -229,7 +246,8 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     P = I.make_peer_partials(wl, device="cuda")
     out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
     send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
-    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"],
+                  **launch.get("opts", {}))
     res = {}
     us = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), steps, warmup, flush, torch)
     st = plan.last_status()
@@ -331,12 +349,18 @@ def run_ablation(args, peaks, flush, torch, E, I):
         send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
 
         def fused(order, n_comm, **opts):
-            plan = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=wl.W - 1, **opts)
-            us = statistics.median(time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), iters, 3, flush, torch))
-            st = plan.last_status()
-            plan.destroy()
-            return {"fused_us": us, "t_gemm_us": st["t_gemm_ns"] / 1e3,
-                    "tail_us": (st["t_end_ns"] - st["t_gemm_ns"]) / 1e3, "n_comm_sms": n_comm}
+            # the slower of the first and the last rank: a collective ends with its slowest rank,
+            # and in the grouped orders a rank's own tiles come early or late in the traversal
+            worst = None
+            for rank in (0, wl.W - 1):
+                plan = E.Plan(wl.M, wl.N, wl.K, wl.W, order, n_comm, rank=rank, **opts)
+                us = statistics.median(time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), iters, 3, flush, torch))
+                st = plan.last_status()
+                plan.destroy()
+                if worst is None or us > worst["fused_us"]:
+                    worst = {"fused_us": us, "t_gemm_us": st["t_gemm_ns"] / 1e3, "slowest_rank": rank,
+                             "tail_us": (st["t_end_ns"] - st["t_gemm_ns"]) / 1e3, "n_comm_sms": n_comm}
+            return worst
 
         def best(order, budgets, **opts):
             return min((fused(order, b, **opts) for b in budgets), key=lambda r: r["fused_us"])
@@ -401,6 +425,7 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "entwine" else args.warmup
 
     from paper_2609_11562_b200 import inputs as I
+    apply_tuned_table()
     wl = I.CONFIGS[args.workload]
     launch = LAUNCH[args.workload]
     if args.impl == "reference":
@@ -451,7 +476,8 @@ def main():
         P = I.make_peer_partials(wl, device="cuda")
         out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
         send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
-        plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+        plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"],
+                  **launch.get("opts", {}))
         plan.gemm_only(A, Bm)
         fn = {"fused": lambda: plan.gemm_rs(A, Bm, P, out, send), "gemm": lambda: plan.gemm_only(A, Bm),
               "comm": lambda: plan.comm_only(None, P, out, send, args.comm_ctas)}[args.kernel_only]
@@ -469,7 +495,8 @@ def main():
     P = I.make_peer_partials(wl, device="cuda")
     out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
     send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
-    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"])
+    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"],
+                  **launch.get("opts", {}))
     sampler.start()
     for _ in range(args.warmup):
         flush.zero_()
@@ -563,6 +590,7 @@ def main():
         "config": {"workload": wl.name, "W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K,
                    "n_comm_sms": launch["n_comm_sms"],
                    "tile_order": "interleaved" if launch["order"] else "row_major",
+                   "plan_options": launch.get("opts", {}),
                    "block": "128x256 blocks on CTA pairs (256x256 pair tiles)",
                    "emulated_rank": launch["rank"], "l2": "flushed between timed steps (512 MiB memset)",
                    "multi_gpu": "replicas only"},

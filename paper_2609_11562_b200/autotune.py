@@ -1,0 +1,202 @@
+"""Offline joint tuner of the fused call's launch configuration (Sec. 3.2 "Communication budget",
+Sec. 4.3: the communication budget, the tile order and the producer's configuration are chosen
+together, by end-to-end latency, once per shape).
+
+For one shape (M, N, K_local, W) the tuner times the fused call over a grid of
+(tile order, n_comm_sms, operand stages, block width BN), keeps the fastest and reports next to
+it the quantities of the paper's budget model: the communication volume of Eq. 2 (here with the
+push traffic of the one-GPU emulation), the computation window T_G of Eq. 3 as measured with the
+chosen budget, and the bandwidth B_req = V / T_G that the consumer side must sustain to finish
+with the producer (Eq. 4), against the bandwidth it reached.
+
+The result is a table keyed by shape that `launch_options` reads back; a shape that is not in
+the table gets the default configuration.  Measuring needs a GPU (there is no CPU fallback);
+reading a table does not.
+
+    python -m paper_2609_11562_b200.autotune --shapes configs --out tuned.json
+"""
+import argparse
+import json
+import os
+import statistics
+
+ORDERS = {"row_major": 0, "interleaved": 1}
+DEFAULT = {"tile_order": "interleaved", "n_comm_sms": 0, "stages": 0, "block_n": 256}
+BUDGETS = (0, 8, 16, 32)
+STAGES = (0, 3, 4, 5)
+
+
+def shape_key(M, N, K_local, W):
+    return f"W{W}_M{M}_N{N}_K{K_local}"
+
+
+def comm_bytes(M, N, W, elem_bytes=2):
+    """Bytes the consumer side moves per call on the emulated rank: every non-owned tile is read
+    and written once (push), every owned tile is read from W contributions and written once
+    (Eq. 2 counts the (W-1)/W * M * N * s bytes that cross the links; the emulation adds the
+    local reads and the writes)."""
+    return M * N * elem_bytes * (3 * W - 1) // W
+
+
+def link_bytes(M, N, W, elem_bytes=2):
+    """Eq. 2: V_comm = (W-1)/W * M * N * s."""
+    return (W - 1) * M * N * elem_bytes // W
+
+
+def b_req(M, N, W, t_gemm_s, elem_bytes=2):
+    """Eq. 4: the bandwidth the communication side must sustain to finish within the
+    computation window, here on the emulation's bytes."""
+    return comm_bytes(M, N, W, elem_bytes) / t_gemm_s
+
+
+def launch_options(table, M, N, K_local, W):
+    """Plan arguments for a shape: (tile_order, n_comm_sms, options dict).  Falls back to the
+    default configuration for a shape the table does not hold."""
+    cfg = dict(DEFAULT)
+    if table:
+        cfg.update(table.get("shapes", {}).get(shape_key(M, N, K_local, W), {}).get("best", {}))
+    opts = {}
+    if cfg["stages"]:
+        opts["stages"] = int(cfg["stages"])
+    if cfg["block_n"] != 256:
+        opts["block_n"] = int(cfg["block_n"])
+    return ORDERS[cfg["tile_order"]], int(cfg["n_comm_sms"]), opts
+
+
+def load_table(path):
+    with open(path) as f:
+        table = json.load(f)
+    if table.get("format") != 1 or "shapes" not in table:
+        raise ValueError(f"{path}: not a tuning table")
+    return table
+
+
+def save_table(table, path):
+    os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+    with open(path, "w") as f:
+        json.dump(table, f, indent=1, sort_keys=True)
+
+
+def _time(fn, flush, torch, iters, warmup=2):
+    for _ in range(warmup):
+        flush.zero_()
+        fn()
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
+
+
+def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=STAGES, ranks=None):
+    """Times the grid on the current CUDA device and returns the table entry of the shape.
+
+    A configuration's latency is the largest over the emulated ranks tried (first, middle, last
+    by default): in the partition-grouped order a rank's own tiles appear early or late in the
+    producer's traversal depending on the rank, and a collective ends with its slowest rank."""
+    import torch
+    from . import entwine as E
+    from . import inputs as I
+    ranks = sorted({0, wl.W // 2, wl.W - 1}) if ranks is None else list(ranks)
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    points = []
+
+    def measure(order_name, n_comm, stg, bn):
+        opts = {}
+        if stg:
+            opts["stages"] = stg
+        if bn != 256:
+            opts["block_n"] = bn
+        worst = None
+        for rank in ranks:
+            try:
+                plan = E.Plan(wl.M, wl.N, wl.K, wl.W, ORDERS[order_name], n_comm, rank=rank, **opts)
+            except E.EntwineError:
+                return None
+            try:
+                us = _time(lambda: plan.gemm_rs(A, Bm, P, out, send), flush, torch, iters)
+                st = plan.last_status()
+            except E.EntwineError:
+                plan.destroy()
+                return None
+            plan.destroy()
+            if worst is None or us > worst["fused_us"]:
+                worst = {"tile_order": order_name, "n_comm_sms": n_comm, "stages": stg, "block_n": bn,
+                         "fused_us": us, "slowest_rank": rank, "t_gemm_us": st["t_gemm_ns"] / 1e3,
+                         "t_end_us": st["t_end_ns"] / 1e3}
+        points.append(worst)
+        return worst
+
+    for order_name in ORDERS:
+        for n_comm in budgets:
+            for stg in stages:
+                measure(order_name, n_comm, stg, 256)
+    best = min(points, key=lambda r: r["fused_us"])
+    if wl.N % 128 == 0:
+        # the narrow producer block with the winner's other settings
+        measure(best["tile_order"], best["n_comm_sms"], best["stages"], 128)
+        best = min(points, key=lambda r: r["fused_us"])
+    t_g = best["t_gemm_us"] * 1e-6
+    tail = (best["t_end_us"] - best["t_gemm_us"]) * 1e-6
+    model = {
+        "link_bytes_eq2": link_bytes(wl.M, wl.N, wl.W),
+        "comm_bytes": comm_bytes(wl.M, wl.N, wl.W),
+        "t_gemm_us_eq3": best["t_gemm_us"],
+        "b_req_GBps_eq4": b_req(wl.M, wl.N, wl.W, t_g) / 1e9,
+        "b_measured_GBps": comm_bytes(wl.M, wl.N, wl.W) / (best["t_end_us"] * 1e-6) / 1e9,
+        "tail_us": tail * 1e6,
+    }
+    default = next(r for r in points if all(r[k] == DEFAULT[k] for k in DEFAULT))
+    del A, Bm, P, out, send
+    torch.cuda.empty_cache()
+    return {"shape": {"W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K},
+            "best": {k: best[k] for k in DEFAULT}, "best_us": best["fused_us"],
+            "default_us": default["fused_us"], "gain_over_default": default["fused_us"] / best["fused_us"],
+            "model": model, "points": points}
+
+
+def tune(workloads, iters=8, keep_points=False):
+    import torch
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # larger than L2
+    table = {"format": 1, "device": torch.cuda.get_device_name(), "shapes": {}}
+    for wl in workloads:
+        entry = tune_shape(wl, flush, iters)
+        if not keep_points:
+            entry.pop("points")
+        table["shapes"][shape_key(wl.M, wl.N, wl.K, wl.W)] = entry
+    return table
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--shapes", default="configs", choices=["configs", "sweep"])
+    ap.add_argument("--out", required=True)
+    ap.add_argument("--iters", type=int, default=8)
+    ap.add_argument("--keep-points", action="store_true")
+    args = ap.parse_args()
+    from . import build as B
+    B.build()
+    from . import inputs as I
+    if args.shapes == "configs":
+        wls = [I.ATTN_OUT, I.MLP_DOWN, I.SHORT_K]
+    else:
+        wls = I.sweep_workloads()
+    table = tune(wls, args.iters, args.keep_points)
+    save_table(table, args.out)
+    for key, e in table["shapes"].items():
+        print(f"{key}: {e['best']} {e['best_us']:.1f} us ({e['gain_over_default']:.3f}x the default), "
+              f"B_req {e['model']['b_req_GBps_eq4']:.0f} GB/s, reached {e['model']['b_measured_GBps']:.0f} GB/s")
+    return 0
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())
