@@ -841,7 +841,10 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
     // ---------------- forward push slots with TMA stores, recycle all slots ----------------
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
     // which is awaited only when kPend younger stores exist or when this thread would idle.
-    constexpr int kPend = 3;
+#ifndef ENTWINE_PEND
+#define ENTWINE_PEND 3
+#endif
+    constexpr int kPend = ENTWINE_PEND;
     // pushed tiles are not read again on this GPU
     const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     unsigned long long pend = 0;  // queue of barrier addresses' slot/ring ids, 8 bits each
