@@ -110,9 +110,10 @@ struct KParams {
   const unsigned* flags_peer;    // [W-1][Q]
   const Task* tasks;
   const int* list_offs;          // [x+1]
-  int* list_head;                // [x]
+  int* list_head;                // [x] head counters of this launch
+  int* list_head_next;           // [x] head counters of the next launch, rewound by this one (or null)
+  StatusSlot* status_next;       // status slot of the next launch, cleared by this one (or null)
   StatusSlot* status;            // [2]
-  unsigned* done_ctr;
 };
 
 // Tensor maps of one launch.  Loads of A and B and the epilogue's stores of C use the
@@ -936,6 +937,22 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   const int stride = PAIR ? P.G / 2 : P.G;
   const int n_my = (is_producer && unit0 < n_units) ? (n_units - unit0 + stride - 1) / stride : 0;
 
+  // Bookkeeping for the NEXT launch, done at the start of this one so that no CTA has anything to
+  // do after its last task: head counters and status slots alternate between two sets, and the
+  // set this launch does not use was last touched by the previous launch, which is complete.
+  if (P.list_head_next) {
+    for (int j = blockIdx.x * kThreads + threadIdx.x; j < P.x; j += gridDim.x * kThreads) P.list_head_next[j] = 0;
+  }
+  if (P.status_next && blockIdx.x == 0 && threadIdx.x == 0) {
+    StatusSlot* nx = P.status_next;
+    nx->code_cta_task = 0;
+    nx->flags_published = 0;
+    nx->tiles_reduced = 0;
+    nx->tiles_pushed = 0;
+    nx->t_start = ~0ULL;
+    nx->t_gemm_end = 0;
+    nx->t_end = 0;
+  }
   if (threadIdx.x == 0) {
     sh.abort = 0;
     sh.blocks_stored = 0;
@@ -1303,25 +1320,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 
   // ---------------- exit bookkeeping ----------------
   __syncthreads();
-  if (threadIdx.x == 0) {
-    atomicMax(&st->t_end, globaltimer_ns());
-    __threadfence();
-    const unsigned prev = atomicAdd(P.done_ctr, 1u);
-    if (prev == gridDim.x - 1) {
-      // last CTA out: rewind the list heads and prepare the other status slot
-      for (int j = 0; j < P.x; ++j) P.list_head[j] = 0;
-      StatusSlot* nx = &P.status[(P.seq & 1) ^ 1];
-      nx->code_cta_task = 0;
-      nx->flags_published = 0;
-      nx->tiles_reduced = 0;
-      nx->tiles_pushed = 0;
-      nx->t_start = ~0ULL;
-      nx->t_gemm_end = 0;
-      nx->t_end = 0;
-      *P.done_ctr = 0;
-      __threadfence();
-    }
-  }
+  if (threadIdx.x == 0) atomicMax(&st->t_end, globaltimer_ns());
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1336,7 +1335,6 @@ struct DeviceState {
   int* list_offs = nullptr;
   int* list_head = nullptr;
   StatusSlot* status = nullptr;
-  unsigned* done_ctr = nullptr;
   unsigned* group_ctr = nullptr;
   unsigned epoch = 0;
   unsigned seq = 0;
@@ -1447,9 +1445,8 @@ static int ensure_device(Plan* p) {
             cudaMalloc(&d->flags_peer, n_peer * 4) == cudaSuccess &&
             cudaMalloc(&d->tasks, t.dev_tasks.size() * sizeof(Task)) == cudaSuccess &&
             cudaMalloc(&d->list_offs, t.list_offs.size() * 4) == cudaSuccess &&
-            cudaMalloc(&d->list_head, size_t(p->x) * 4) == cudaSuccess &&
+            cudaMalloc(&d->list_head, size_t(p->x) * 2 * 4) == cudaSuccess &&
             cudaMalloc(&d->status, 2 * sizeof(StatusSlot)) == cudaSuccess &&
-            cudaMalloc(&d->done_ctr, 4) == cudaSuccess &&
             cudaMalloc(&d->group_ctr, size_t(g.P_blk) * 4) == cudaSuccess;
   if (ok) {
     StatusSlot init[2];
@@ -1462,9 +1459,8 @@ static int ensure_device(Plan* p) {
                     cudaMemcpyHostToDevice) == cudaSuccess &&
          cudaMemcpy(d->list_offs, t.list_offs.data(), t.list_offs.size() * 4, cudaMemcpyHostToDevice) ==
              cudaSuccess &&
-         cudaMemset(d->list_head, 0, size_t(p->x) * 4) == cudaSuccess &&
+         cudaMemset(d->list_head, 0, size_t(p->x) * 2 * 4) == cudaSuccess &&
          cudaMemcpy(d->status, init, sizeof(init), cudaMemcpyHostToDevice) == cudaSuccess &&
-         cudaMemset(d->done_ctr, 0, 4) == cudaSuccess &&
          cudaMemset(d->group_ctr, 0, size_t(g.P_blk) * 4) == cudaSuccess;
   }
   p->dev = d;
@@ -1491,7 +1487,6 @@ void device_release(Plan* p) {
   cudaFree(d->list_offs);
   cudaFree(d->list_head);
   cudaFree(d->status);
-  cudaFree(d->done_ctr);
   cudaFree(d->group_ctr);
   cudaFree(d->sA);
   cudaFree(d->sB);
@@ -1637,8 +1632,13 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.group_ctr = d->group_ctr;
   kp.claim = claim_size(g.W);
   kp.epoch = d->epoch;
-  d->seq += 1;
-  kp.seq = d->seq;
+  // the launch number is committed only when the launch has been enqueued
+  const unsigned seq_next = d->seq + 1;
+  kp.seq = seq_next;
+  // two sets of head counters and status slots, used alternately; a launch rewinds the other set
+  kp.list_head = d->list_head + size_t(seq_next & 1) * p->x;
+  kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * p->x;
+  kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
   rc = ring_geometry(p, &kp);
   if (rc != ENTWINE_OK) return rc;
@@ -1650,9 +1650,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.flags_peer = d->flags_peer;
   kp.tasks = d->tasks;
   kp.list_offs = d->list_offs;
-  kp.list_head = d->list_head;
   kp.status = d->status;
-  kp.done_ctr = d->done_ctr;
 
   int grid;
   const bool pair = p->pair;
@@ -1707,6 +1705,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   else if (g.BN == 256) rc = launch_bn<256, false>(p, kp, maps, grid, stream);
   else rc = launch_bn<128, false>(p, kp, maps, grid, stream);
   if (rc != ENTWINE_OK) return rc;
+  d->seq = seq_next;
   p->launched = true;
   d->last_stream = stream;
   d->status_pending = true;
@@ -1769,8 +1768,7 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]) {
   out[7] = (s.t_end > s.t_start) ? int64_t(s.t_end - s.t_start) : 0;
   if (code) {
     // the launch gave up part-way: rewind what its last CTA would have rewound
-    cudaMemset(d->list_head, 0, size_t(plan->x) * 4);
-    cudaMemset(d->done_ctr, 0, 4);
+    cudaMemset(d->list_head, 0, size_t(plan->x) * 2 * 4);
     StatusSlot init[2];
     std::memset(init, 0, sizeof(init));
     init[0].t_start = init[1].t_start = ~0ULL;
@@ -1929,8 +1927,9 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out_shard);
   kp.status = reinterpret_cast<StatusSlot*>(ctrl + off_status);
-  kp.done_ctr = reinterpret_cast<unsigned*>(ctrl + off_done);
   kp.list_head = reinterpret_cast<int*>(ctrl + off_heads);
+  kp.list_head_next = nullptr;  // this entry point clears its control block before every launch
+  kp.status_next = nullptr;
   kp.list_offs = reinterpret_cast<const int*>(ctrl + off_offs);
   kp.flags_own = reinterpret_cast<unsigned*>(ctrl + off_fown);
   kp.flags_peer = reinterpret_cast<const unsigned*>(ctrl + off_fpeer);
