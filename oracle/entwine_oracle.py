@@ -34,6 +34,11 @@ Parity status of each function (what pins it is in tests/test_oracle_*.py):
   bf16_round                       pinned: hand-computed ties, torch's conversion
   staged_model                     diagnostic; pinned against reduce_scatter_ref within
                                    the rounding bound derived in its docstring
+  rmsnorm_ref, layer_chain_ref     pinned: closed forms (constant rows, one-hot rows, scale
+                                   invariance at eps = 0), torch's rms_norm in float64
+  norm_task_order                  parity unpinned by the paper (the paper evaluates the
+                                   operator chain of Sec. 5.2.3 but does not fuse it; the
+                                   band rule is this build's design, see its docstring)
 """
 from __future__ import annotations
 
@@ -386,6 +391,38 @@ def staged_model(A_bits, B_bits, peers_bits, r: int, W: int):
     out = bf16_round(acc.astype(np.float64))
     send = np.stack([Cb[d * R:(d + 1) * R] for d in range(W) if d != r])
     return out, send
+
+
+# --------------------------------------------------------------------------------------
+# layer-level chain: ReduceScatter -> residual add -> RMSNorm (Sec. 5.2.3)
+# --------------------------------------------------------------------------------------
+def rmsnorm_ref(h: np.ndarray, weight: np.ndarray, eps: float) -> np.ndarray:
+    """RMSNorm over the last axis, float64: h / sqrt(mean(h^2) + eps) * weight."""
+    h = np.asarray(h, np.float64)
+    ms = np.mean(h * h, axis=-1, keepdims=True)
+    return h / np.sqrt(ms + eps) * np.asarray(weight, np.float64)
+
+
+def layer_chain_ref(ref_out: np.ndarray, residual_bits: np.ndarray, weight_bits: np.ndarray,
+                    eps: float):
+    """The operator chain that follows the ReduceScatter in the attention-output layer
+    (Sec. 5.2.3): hidden = reduce-scattered output + residual; normed = RMSNorm(hidden).
+
+    ref_out [R,N] float64 (reduce_scatter_ref); residual [R,N] and weight [N] as bf16 bits.
+    Returns (hidden, normed) in float64, the definition with no intermediate rounding.
+    """
+    hidden = ref_out + bf16_bits_to_f64(residual_bits)
+    return hidden, rmsnorm_ref(hidden, bf16_bits_to_f64(weight_bits), eps)
+
+
+def norm_task_order(M: int, N: int, W: int):
+    """Normalisation tasks of the emulated rank in the order they are handed out: one per
+    128 x 128 tile of the rank's partition, tile row (a band of 128 complete rows) by tile
+    row, tile column fastest.  A band's tasks may run once all nTn tiles of the band are
+    reduced.  Returns int32 [Q, 2] of (band, tile column)."""
+    rowsT = M // W // T
+    nTn = N // T
+    return np.array([(b, tc) for b in range(rowsT) for tc in range(nTn)], np.int32).reshape(-1, 2)
 
 
 # --------------------------------------------------------------------------------------

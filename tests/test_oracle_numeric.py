@@ -182,3 +182,51 @@ def test_input_generators_are_seeded_and_shaped():
     assert 0.9 < P.float().std() < 1.1
     assert len(I.sweep_workloads()) == 60
     assert I.ATTN_OUT.comm_bytes == 4096 * 4096 * 2 * 11 // 4
+
+
+def test_rmsnorm_closed_forms_and_library():
+    """RMSNorm definition: constant rows normalise to sign * weight; a one-hot row of value v
+    in N columns gives sqrt(N) * sign(v) * w at that column; scale invariance at eps = 0;
+    float64 torch.nn.functional.rms_norm as the library routine."""
+    rng = np.random.default_rng(5)
+    N = 96
+    w = rng.normal(size=N)
+    const = np.full((3, N), -2.5)
+    assert np.allclose(O.rmsnorm_ref(const, w, 0.0), -w[None, :].repeat(3, 0), rtol=1e-14)
+    onehot = np.zeros((2, N))
+    onehot[0, 7], onehot[1, 40] = 3.0, -0.25
+    got = O.rmsnorm_ref(onehot, w, 0.0)
+    assert np.isclose(got[0, 7], np.sqrt(N) * w[7]) and np.isclose(got[1, 40], -np.sqrt(N) * w[40])
+    assert np.count_nonzero(got) == 2
+    h = rng.normal(size=(5, N))
+    assert np.allclose(O.rmsnorm_ref(h, w, 0.0), O.rmsnorm_ref(1e3 * h, w, 0.0), rtol=1e-12)
+    # eps matters exactly as mean(h^2) + eps
+    eps = 0.37
+    manual = h / np.sqrt((h ** 2).sum(-1, keepdims=True) / N + eps) * w
+    assert np.allclose(O.rmsnorm_ref(h, w, eps), manual, rtol=1e-14)
+    lib = torch.nn.functional.rms_norm(torch.from_numpy(h), (N,), torch.from_numpy(w), eps).numpy()
+    assert np.allclose(O.rmsnorm_ref(h, w, eps), lib, rtol=1e-12, atol=1e-14)
+
+
+def test_layer_chain_is_residual_add_then_rmsnorm():
+    rng = np.random.default_rng(6)
+    R, N = 8, 64
+    out = rng.normal(size=(R, N))
+    res_bits = O.f64_to_bf16_bits(rng.normal(size=(R, N)))
+    w_bits = O.f64_to_bf16_bits(1.0 + 0.1 * rng.normal(size=N))
+    hidden, normed = O.layer_chain_ref(out, res_bits, w_bits, 1e-5)
+    res, w = O.bf16_bits_to_f64(res_bits), O.bf16_bits_to_f64(w_bits)
+    assert np.array_equal(hidden, out + res)
+    for i in range(R):  # row by row, written out
+        ms = sum(float(v) ** 2 for v in hidden[i]) / N
+        assert np.allclose(normed[i], hidden[i] / np.sqrt(ms + 1e-5) * w, rtol=1e-13)
+    # zero residual and unit weight: rows of unit RMS
+    _, n1 = O.layer_chain_ref(out, np.zeros((R, N), np.uint16), O.f64_to_bf16_bits(np.ones(N)), 0.0)
+    assert np.allclose((n1 ** 2).mean(-1), 1.0, rtol=1e-12)
+
+
+def test_norm_task_order_covers_every_tile_band_by_band():
+    order = O.norm_task_order(1024, 768, 4)
+    rowsT, nTn = 1024 // 4 // 128, 768 // 128
+    assert order.shape == (rowsT * nTn, 2)
+    assert [tuple(v) for v in order] == [(b, c) for b in range(rowsT) for c in range(nTn)]
