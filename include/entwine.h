@@ -183,6 +183,26 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B,
                          const void* peer_partials, void* out_shard, void* send_bufs);
 
 /*
+ * entwine_gemm_rs_norm - the fused call followed, inside the same launch, by the rest of the
+ * attention-output layer's chain (Sec. 5.2.3: GEMM + ReduceScatter, then residual addition and
+ * RMSNorm).  The reduction of an owned tile adds residual[R][N] to the rank-order fp32 sum and
+ * rounds once: hidden_out[R][N] (bf16) is the new residual stream and takes the place of
+ * out_shard.  When all tiles of a band of 128 rows are reduced the band's rows are complete,
+ * and its tiles are normalised by whichever CTAs are free:
+ *   norm_out[i][j] = bf16( hidden_out[i][j] * rsqrt(mean_j(hidden_out[i][:]^2) + eps) * weight[j] ),
+ * computed in fp32 from the stored bf16 hidden values (row sums of squares are accumulated in a
+ * fixed order: results are bitwise reproducible).  send_bufs as in entwine_gemm_rs.
+ * residual, weight[N], hidden_out, norm_out: device pointers, bf16, 16-byte aligned; eps >= 0.
+ * Errors as entwine_gemm_rs; ENTWINE_ERR_INVALID also if the plan has more consumer lists than
+ * consumer CTAs (ENTWINE_OPT_LISTS).  Not available through the host-buffer or the
+ * no-allocation entry points.
+ */
+int entwine_gemm_rs_norm(entwine_plan_t plan, const void* A, const void* B,
+                         const void* peer_partials, const void* residual, const void* weight,
+                         float eps, void* hidden_out, void* norm_out, void* send_bufs,
+                         void* stream);
+
+/*
  * entwine_gemm_only - the producer alone on all SMs (no consumer work): fills the plan's
  * partial-output workspace and publishes the flags.  Gives the uncontended GEMM time of the
  * overlap-efficiency ratio (Sec. 5.2.1, App. C).  A, B device pointers.

@@ -110,7 +110,15 @@ struct KParams {
   const unsigned* flags_peer;    // [W-1][Q]
   const Task* tasks;
   const int* list_offs;          // [x+1]
-  int* list_head;                // [x] head counters of this launch
+  // layer chain (residual add + RMSNorm fused into the consumer), off unless norm != 0
+  int norm;
+  float eps;
+  const __nv_bfloat16* residual;  // [R][N]
+  const __nv_bfloat16* weight;    // [N]
+  __nv_bfloat16* norm_out;        // [R][N]
+  float* ssq_part;                // [R][nTn] sum of squares of a row's 128 elements inside one tile
+  unsigned* band_ctr;             // [rowsT] reduced tiles per band of 128 rows (cleared per launch)
+  int* list_head;                // [x + 1] head counters of this launch; entry x: normalisation tasks
   int* list_head_next;           // [x] head counters of the next launch, rewound by this one (or null)
   StatusSlot* status_next;       // status slot of the next launch, cleared by this one (or null)
   StatusSlot* status;            // [2]
@@ -427,14 +435,16 @@ __device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) 
 // status helpers
 // ------------------------------------------------------------------------------------------
 struct SlotMeta {
-  int kind;      // 0 reduce step, 1 push step, -1 end of work, -2 continue on ring B
+  int kind;      // 0 reduce step, 1 push step, 2 normalisation of a tile, -1 end of work, -2 continue on ring B
   int dst_x;     // column of the destination box
   int dst_y;     // row of the destination box in the destination buffer
+  int aux;       // layer chain: band (tile row) whose count the last step of a reduce task raises, else -1
 };
 struct CtaShared {
   volatile int abort;      // a role of this CTA (or another CTA) gave up
   volatile int gemm_done;  // this CTA's producer work is over; its shared memory is free
   int blocks_stored;       // blocks of this CTA whose partial-C stores are complete
+  float inv_rms[kTile];    // layer chain: 1 / RMS of the rows of the tile being normalised
   SlotMeta meta[2][kMaxSlots];
 };
 
@@ -477,6 +487,21 @@ __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
       else if (now - t0 > P.wait_budget_ns) return false;
     }
     __nanosleep(64);  // longer, growing pauses (up to 4 us) were measured: no effect on the producer
+  }
+}
+
+// Bounded acquire-poll of a counter until it reaches `target`.
+__device__ __forceinline__ bool wait_count(const unsigned* f, unsigned target, const KParams& P) {
+  unsigned long long t0 = 0;
+  for (uint32_t spins = 1;; ++spins) {
+    if (ld_acquire_gpu(f) >= target) return true;
+    if ((spins % 32) == 0) {
+      if (global_abort(P)) return false;
+      unsigned long long now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > P.wait_budget_ns) return false;
+    }
+    __nanosleep(128);
   }
 }
 
@@ -738,6 +763,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
               m.kind = kind;
               m.dst_x = col;
               m.dst_y = dst_row + step * rows;
+              m.aux = (P.norm && kind == 0 && step == n_steps - 1) ? dst_row / kTile : -1;
               mbar_arrive_expect_tx(ring.full(slot), tx);
               // Few, large TMA operations: the per-operation cost of the TMA unit, not bandwidth,
               // bounds a consumer that issues many small boxes.
@@ -787,6 +813,49 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
       }
       if (!any) break;
     }
+    // Layer chain: when no reduce or push task is left to claim, the CTAs share the normalisation
+    // tasks (one per tile of the rank's partition, band by band) through one counter.  A task
+    // waits until all nTn tiles of its band are reduced; the reducing warps read the band from
+    // L2 themselves, the ring slot only hands them the task.
+    if (P.norm && ok && n_lists > 0) {
+      int* head = &P.list_head[P.x];
+      int c0 = P.Q, c1 = P.Q;
+      if (lane == 0) {
+        c0 = atomicAdd(head, 1);
+        c1 = atomicAdd(head, 1);
+      }
+      while (ok) {
+        const int i = __shfl_sync(0xffffffffu, c0, 0);
+        if (i >= P.Q) break;
+        c0 = c1;
+        if (lane == 0) c1 = atomicAdd(head, 1);
+        const int band = i / P.nTn, tc = i - band * P.nTn;
+        bool band_ok = true;
+        if (lane == 0) band_ok = wait_count(&P.band_ctr[band], (unsigned)P.nTn, P);
+        ok = __all_sync(0xffffffffu, band_ok);
+        if (!ok) {
+          if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, -7);
+          break;
+        }
+        maybe_switch();
+        if (!ok) break;
+        bool free_slot = true;
+        if (lane == 0) {
+          const int slot = it % ring.n_slots;
+          free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+          if (free_slot) {
+            SlotMeta& m = sh->meta[ring.id][slot];
+            m.kind = 2;
+            m.dst_x = tc * kTile;
+            m.dst_y = band * kTile;
+            m.aux = -1;
+            mbar_arrive(ring.full(slot));
+          }
+        }
+        ok = __all_sync(0xffffffffu, free_slot);
+        it += 1;
+      }
+    }
     // end-of-work marker so that the other consumer warps leave their loops
     if (lane == 0) {
       const int slot = it % ring.n_slots;
@@ -818,7 +887,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         ph = 0;
         continue;
       }
-      if (m.kind == 0) {
+      if (m.kind == 0 && !P.norm) {
         const uint32_t sbase = ring.base + slot * ring.slot_bytes;
         const int rs = ring.rs, sub_bytes = ring.sub_bytes;
         __nv_bfloat16* dst = P.out + (long long)m.dst_y * P.N + m.dst_x;
@@ -832,6 +901,63 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
           for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
           __stcs(reinterpret_cast<uint4*>(dst + (long long)(c >> 4) * P.N + (c & 15) * 8), pack_bf16x8(a));
         }
+      } else if (m.kind == 0) {
+        // Layer chain (Sec. 5.2.3): the same rank-order fp32 sum, plus the residual; the bf16
+        // result is the new residual stream (written to P.out), and the sum of squares of the
+        // 128 stored values of each row inside this tile goes to ssq_part (one writer each).
+        const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
+        const int n_chunks = rs * (kTile * 2 / 16);
+        for (int c0 = 0; c0 < n_chunks; c0 += kRedThreads) {
+          const int c = c0 + ctid;
+          const bool act = c < n_chunks;
+          float ssq = 0.f;
+          if (act) {
+            const long long off = (long long)(m.dst_y + (c >> 4)) * P.N + m.dst_x + (c & 15) * 8;
+            const uint4 res = __ldcs(reinterpret_cast<const uint4*>(P.residual + off));
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            const uint32_t addr = sbase + c * 16;
+            acc_bf16x8(a, ld_shared_v4(addr));
+#pragma unroll 4
+            for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
+            acc_bf16x8(a, res);
+            const uint4 o = pack_bf16x8(a);
+            __stcg(reinterpret_cast<uint4*>(P.out + off), o);  // re-read from L2 by the normalisation
+            float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            acc_bf16x8(h, o);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ssq = fmaf(h[e], h[e], ssq);
+          }
+          // the 16 threads of a row segment (half a warp) add up in a fixed order
+#pragma unroll
+          for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
+          if (act && (lane & 15) == 0)
+            __stcg(&P.ssq_part[(long long)(m.dst_y + (c >> 4)) * P.nTn + m.dst_x / kTile], ssq);
+        }
+      } else if (m.kind == 2) {
+        // Normalisation of one 128 x 128 tile of a complete band: 1/RMS of each of its rows from
+        // the nTn partial sums (fixed order), then hidden * inv_rms * weight, rounded once.
+        if (ctid < kTile) {
+          const float* pr = P.ssq_part + (long long)(m.dst_y + ctid) * P.nTn;
+          float sum = 0.f;
+          for (int tc = 0; tc < P.nTn; ++tc) sum += __ldcg(pr + tc);
+          sh->inv_rms[ctid] = rsqrtf(sum / (float)P.N + P.eps);
+        }
+        named_bar_sync(2, kRedThreads);
+        float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        acc_bf16x8(w, __ldg(reinterpret_cast<const uint4*>(P.weight + m.dst_x + (ctid & 15) * 8)));
+#pragma unroll 4
+        for (int c = ctid; c < kTile * (kTile * 2 / 16); c += kRedThreads) {
+          const int row = c >> 4;
+          const long long off = (long long)(m.dst_y + row) * P.N + m.dst_x + (c & 15) * 8;
+          float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          acc_bf16x8(h, __ldcg(reinterpret_cast<const uint4*>(P.out + off)));
+          const float inv = sh->inv_rms[row];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[e] = h[e] * inv * w[e];
+          __stcs(reinterpret_cast<uint4*>(P.norm_out + off), pack_bf16x8(h));
+        }
+        named_bar_sync(2, kRedThreads);  // inv_rms is rewritten by the next normalisation step
       }
       // one arrival per warp returns the slot (a push step is forwarded by the store warp alone;
       // the arrival then only says that this warp has read the slot's header)
@@ -842,10 +968,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
     // ---------------- forward push slots with TMA stores, recycle all slots ----------------
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
     // which is awaited only when kPend younger stores exist or when this thread would idle.
-#ifndef ENTWINE_PEND
-#define ENTWINE_PEND 3
-#endif
-    constexpr int kPend = ENTWINE_PEND;
+    constexpr int kPend = 3;
     // pushed tiles are not read again on this GPU
     const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     unsigned long long pend = 0;  // queue of barrier addresses' slot/ring ids, 8 bits each
@@ -883,7 +1006,12 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         sh->abort = 1;
         break;
       }
-      if (m.kind == 0) {
+      if (m.kind == 0 || m.kind == 2) {
+        if (m.aux >= 0) {
+          // layer chain: the last step of a reduce task counts its tile in the band
+          fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
+          atomicAdd(&P.band_ctr[m.aux], 1u);
+        }
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
         tma_store_2d_hint(&maps.send_st[ring.geom], m.dst_x, m.dst_y, sbase, pol);
@@ -941,7 +1069,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   // do after its last task: head counters and status slots alternate between two sets, and the
   // set this launch does not use was last touched by the previous launch, which is complete.
   if (P.list_head_next) {
-    for (int j = blockIdx.x * kThreads + threadIdx.x; j < P.x; j += gridDim.x * kThreads) P.list_head_next[j] = 0;
+    for (int j = blockIdx.x * kThreads + threadIdx.x; j <= P.x; j += gridDim.x * kThreads) P.list_head_next[j] = 0;
   }
   if (P.status_next && blockIdx.x == 0 && threadIdx.x == 0) {
     StatusSlot* nx = P.status_next;
@@ -1336,6 +1464,8 @@ struct DeviceState {
   int* list_head = nullptr;
   StatusSlot* status = nullptr;
   unsigned* group_ctr = nullptr;
+  float* ssq_part = nullptr;     // layer chain: [R][nTn]
+  unsigned* band_ctr = nullptr;  // layer chain: [rowsT]
   unsigned epoch = 0;
   unsigned seq = 0;
   bool status_pending = false;
@@ -1445,7 +1575,7 @@ static int ensure_device(Plan* p) {
             cudaMalloc(&d->flags_peer, n_peer * 4) == cudaSuccess &&
             cudaMalloc(&d->tasks, t.dev_tasks.size() * sizeof(Task)) == cudaSuccess &&
             cudaMalloc(&d->list_offs, t.list_offs.size() * 4) == cudaSuccess &&
-            cudaMalloc(&d->list_head, size_t(p->x) * 2 * 4) == cudaSuccess &&
+            cudaMalloc(&d->list_head, size_t(p->x + 1) * 2 * 4) == cudaSuccess &&
             cudaMalloc(&d->status, 2 * sizeof(StatusSlot)) == cudaSuccess &&
             cudaMalloc(&d->group_ctr, size_t(g.P_blk) * 4) == cudaSuccess;
   if (ok) {
@@ -1459,7 +1589,7 @@ static int ensure_device(Plan* p) {
                     cudaMemcpyHostToDevice) == cudaSuccess &&
          cudaMemcpy(d->list_offs, t.list_offs.data(), t.list_offs.size() * 4, cudaMemcpyHostToDevice) ==
              cudaSuccess &&
-         cudaMemset(d->list_head, 0, size_t(p->x) * 2 * 4) == cudaSuccess &&
+         cudaMemset(d->list_head, 0, size_t(p->x + 1) * 2 * 4) == cudaSuccess &&
          cudaMemcpy(d->status, init, sizeof(init), cudaMemcpyHostToDevice) == cudaSuccess &&
          cudaMemset(d->group_ctr, 0, size_t(g.P_blk) * 4) == cudaSuccess;
   }
@@ -1488,6 +1618,8 @@ void device_release(Plan* p) {
   cudaFree(d->list_head);
   cudaFree(d->status);
   cudaFree(d->group_ctr);
+  cudaFree(d->ssq_part);
+  cudaFree(d->band_ctr);
   cudaFree(d->sA);
   cudaFree(d->sB);
   cudaFree(d->sPeers);
@@ -1579,12 +1711,35 @@ static int ring_geometry(const Plan* p, KParams* kp) {
 }
 
 // Common launch path.  `partial` overrides the workspace in consumer-only mode.
+// Arguments of the layer chain (residual add + RMSNorm after the reduction).
+struct NormArgs {
+  const void* residual;  // [R][N] bf16
+  const void* weight;    // [N] bf16
+  void* norm_out;        // [R][N] bf16
+  float eps;
+};
+
 static int launch(Plan* p, int mode, const void* A, const void* B, const void* partial, const void* peers,
-                  void* out, void* send, int n_ctas, cudaStream_t stream) {
+                  void* out, void* send, int n_ctas, cudaStream_t stream, const NormArgs* norm = nullptr) {
   int rc = ensure_device(p);
   if (rc != ENTWINE_OK) return rc;
   DeviceState* d = p->dev;
   const Geometry& g = p->g;
+  if (norm) {
+    if (mode != MODE_FUSED || !norm->residual || !norm->weight || !norm->norm_out ||
+        !aligned16(norm->residual) || !aligned16(norm->weight) || !aligned16(norm->norm_out) ||
+        !(norm->eps >= 0.f))
+      return ENTWINE_ERR_INVALID;
+    // a CTA that waits for a band cannot drain lists: every list needs a consumer CTA of its own
+    if (p->x > p->n_gemm_ctas + p->n_comm_ctas) return ENTWINE_ERR_INVALID;
+    if (!d->ssq_part) {
+      if (cudaMalloc(&d->ssq_part, size_t(g.R) * g.nTn * 4) != cudaSuccess ||
+          cudaMalloc(&d->band_ctr, size_t(g.rowsT) * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return ENTWINE_ERR_CUDA;
+      }
+    }
+  }
   if (mode != MODE_COMM_ONLY && (!A || !B || !aligned16(A) || !aligned16(B))) return ENTWINE_ERR_INVALID;
   if (mode != MODE_GEMM_ONLY &&
       (!peers || !out || !send || !aligned16(peers) || !aligned16(out) || !aligned16(send)))
@@ -1630,14 +1785,24 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.skip_wait = (mode == MODE_COMM_ONLY) ? 1 : 0;
   kp.release_group = p->release_group;
   kp.group_ctr = d->group_ctr;
+  kp.norm = norm ? 1 : 0;
+  if (norm) {
+    kp.eps = norm->eps;
+    kp.residual = static_cast<const __nv_bfloat16*>(norm->residual);
+    kp.weight = static_cast<const __nv_bfloat16*>(norm->weight);
+    kp.norm_out = static_cast<__nv_bfloat16*>(norm->norm_out);
+    kp.ssq_part = d->ssq_part;
+    kp.band_ctr = d->band_ctr;
+    CK(cudaMemsetAsync(d->band_ctr, 0, size_t(g.rowsT) * 4, stream));
+  }
   kp.claim = claim_size(g.W);
   kp.epoch = d->epoch;
   // the launch number is committed only when the launch has been enqueued
   const unsigned seq_next = d->seq + 1;
   kp.seq = seq_next;
   // two sets of head counters and status slots, used alternately; a launch rewinds the other set
-  kp.list_head = d->list_head + size_t(seq_next & 1) * p->x;
-  kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * p->x;
+  kp.list_head = d->list_head + size_t(seq_next & 1) * (p->x + 1);
+  kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
   rc = ring_geometry(p, &kp);
@@ -1725,6 +1890,19 @@ int entwine_gemm_rs(entwine_plan_t plan, const void* A, const void* B, const voi
                 static_cast<cudaStream_t>(stream));
 }
 
+int entwine_gemm_rs_norm(entwine_plan_t plan, const void* A, const void* B, const void* peer_partials,
+                         const void* residual, const void* weight, float eps, void* hidden_out,
+                         void* norm_out, void* send_bufs, void* stream) {
+  if (!plan) return ENTWINE_ERR_INVALID;
+  NormArgs na;
+  na.residual = residual;
+  na.weight = weight;
+  na.norm_out = norm_out;
+  na.eps = eps;
+  return launch(plan, MODE_FUSED, A, B, nullptr, peer_partials, hidden_out, send_bufs, 0,
+                static_cast<cudaStream_t>(stream), &na);
+}
+
 int entwine_gemm_only(entwine_plan_t plan, const void* A, const void* B, void* stream) {
   if (!plan) return ENTWINE_ERR_INVALID;
   return launch(plan, MODE_GEMM_ONLY, A, B, nullptr, nullptr, nullptr, nullptr, 0,
@@ -1768,7 +1946,7 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]) {
   out[7] = (s.t_end > s.t_start) ? int64_t(s.t_end - s.t_start) : 0;
   if (code) {
     // the launch gave up part-way: rewind what its last CTA would have rewound
-    cudaMemset(d->list_head, 0, size_t(plan->x) * 2 * 4);
+    cudaMemset(d->list_head, 0, size_t(plan->x + 1) * 2 * 4);
     StatusSlot init[2];
     std::memset(init, 0, sizeof(init));
     init[0].t_start = init[1].t_start = ~0ULL;
@@ -1914,6 +2092,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.skip_wait = 0;
   kp.release_group = 1;  // this entry point keeps the per-block release
   kp.group_ctr = nullptr;
+  kp.norm = 0;
   kp.claim = claim_size(g.W);
   kp.epoch = 1;  // the flags were cleared above
   kp.seq = 0;

@@ -33,11 +33,13 @@ RELEASE_PARTITION, RELEASE_WHOLE = -1, -2
 # every symbol include/entwine.h declares
 SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gemm_rs_host",
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
-           "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static")
+           "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static",
+           "entwine_gemm_rs_norm")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
 _lib.entwine_set_option.argtypes = [_vp, _int, _i64]
+_lib.entwine_gemm_rs_norm.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
 _lib.entwine_gemm_rs.argtypes = [_vp] * 7
 _lib.entwine_gemm_rs_host.argtypes = [_vp] * 6
 _lib.entwine_gemm_only.argtypes = [_vp] * 4
@@ -116,6 +118,12 @@ class Plan:
     def gemm_rs(self, A, B, peer_partials, out_shard, send_bufs, stream=None):
         _check(_lib.entwine_gemm_rs(self._h, _ptr(A), _ptr(B), _ptr(peer_partials), _ptr(out_shard),
                                     _ptr(send_bufs), _stream(stream)), "entwine_gemm_rs")
+
+    def gemm_rs_norm(self, A, B, peer_partials, residual, weight, eps, hidden_out, norm_out, send_bufs,
+                     stream=None):
+        _check(_lib.entwine_gemm_rs_norm(self._h, _ptr(A), _ptr(B), _ptr(peer_partials), _ptr(residual),
+                                         _ptr(weight), float(eps), _ptr(hidden_out), _ptr(norm_out),
+                                         _ptr(send_bufs), _stream(stream)), "entwine_gemm_rs_norm")
 
     def gemm_rs_host(self, A, B, peer_partials, out_shard, send_bufs):
         """Host tensors (CPU, bf16, contiguous; pinned for speed)."""

@@ -130,6 +130,17 @@ def make_peer_partials(wl: Workload, device="cpu", seed_offset: int = 0) -> torc
     return out
 
 
+def make_layer_inputs(wl: Workload, device="cpu"):
+    """Inputs of the layer chain that follows the reduction: the residual stream [R, N] ~ N(0,1)
+    and the RMSNorm weight [N] ~ 1 + 0.1 N(0,1), bf16, streams of their own."""
+    s = wl.seed
+    res = torch.randn(wl.R, wl.N, generator=_gen(s * 16 + 11, device), device=device,
+                      dtype=torch.float32).to(torch.bfloat16)
+    w = (1.0 + 0.1 * torch.randn(wl.N, generator=_gen(s * 16 + 12, device), device=device,
+                                 dtype=torch.float32)).to(torch.bfloat16)
+    return res, w
+
+
 def bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns on the host (what the oracle consumes)."""
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view("uint16")
