@@ -398,6 +398,73 @@ def run_ablation(args, peaks, flush, torch, E, I):
     return 0
 
 
+def run_layer_chain(args, peaks, flush, torch, E, I):
+    """Layer-level chain of Sec. 5.2.3: the attention output of a Llama-3-70B-shaped layer at
+    TP = 8 (hidden 8192, K_local = 1024): GEMM + ReduceScatter, residual addition, RMSNorm, at
+    three sequence lengths.  One launch (entwine_gemm_rs_norm) against the fused GEMM-RS
+    followed by library kernels for the rest, and against the fully unfused sequence."""
+    import torch.nn.functional as F
+    iters = max(args.sweep_iters, 10)
+    report = {}
+    for seq in (4096, 8192, 16384):
+        wl = I.Workload(f"layer_seq{seq}", 8, seq, 8192, 1024, "normal", "normal_total_fanin", 7, seq // 4096)
+        A, Bm = I.make_operands(wl, device="cuda")
+        P = I.make_peer_partials(wl, device="cuda")
+        res, w = I.make_layer_inputs(wl, device="cuda")
+        hidden = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        normed = torch.empty_like(hidden)
+        out = torch.empty_like(hidden)
+        send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+        Cfull = torch.empty(wl.M, wl.N, dtype=torch.bfloat16, device="cuda")
+        plan = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=wl.W - 1)
+        med = statistics.median
+
+        def rest():
+            h = out + res
+            return h, F.rms_norm(h, (wl.N,), w, 1e-5)
+
+        def fused_then_library():
+            plan.gemm_rs(A, Bm, P, out, send)
+            return rest()
+
+        def unfused():
+            torch.matmul(A, Bm.t(), out=Cfull)
+            plan.comm_only(Cfull, P, out, send, 0)
+            return rest()
+
+        one = med(time_steps(lambda: plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send),
+                             iters, 3, flush, torch))
+        st = plan.last_status()
+        two = med(time_steps(fused_then_library, iters, 3, flush, torch))
+        plan.last_status()
+        three = med(time_steps(unfused, iters, 3, flush, torch))
+        plan.last_status()
+        rs_only = med(time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), iters, 3, flush, torch))
+        plan.last_status()
+        # same numbers as the library chain applied to this launch's hidden stream
+        plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send)
+        plan.last_status()
+        lib = F.rms_norm(hidden, (wl.N,), w, 1e-5)
+        max_ulp_diff = float(((normed.float() - lib.float()).abs() / lib.float().abs().clamp_min(1e-3)).max())
+        plan.destroy()
+        report[f"seq_{seq}"] = {
+            "shape": {"W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K},
+            "one_launch_us": one, "gemm_rs_then_library_add_norm_us": two,
+            "cublas_reduce_add_norm_us": three, "gemm_rs_alone_us": rs_only,
+            "speedup_vs_gemm_rs_then_library": two / one, "speedup_vs_unfused": three / one,
+            "chain_cost_over_gemm_rs_us": one - rs_only,
+            "t_gemm_us": st["t_gemm_ns"] / 1e3, "t_end_us": st["t_end_ns"] / 1e3,
+            "max_rel_diff_vs_library_rms_norm": max_ulp_diff,
+        }
+        del A, Bm, P, res, w, hidden, normed, out, send, Cfull
+        torch.cuda.empty_cache()
+    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+    with open(os.path.join(ROOT, "gpurun_out", "layer_chain.json"), "w") as f:
+        json.dump(report, f, indent=1)
+    print(json.dumps({"layer_chain": report}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -415,6 +482,9 @@ def main():
     ap.add_argument("--ablation", action="store_true",
                     help="the design ablations (computation order, release granularity, SM sharing) on a "
                          "short-K and a long-K shape; prints one JSON line and writes gpurun_out/ablation.json")
+    ap.add_argument("--layer-chain", action="store_true",
+                    help="GEMM-RS + residual add + RMSNorm in one launch against library kernels for the rest "
+                         "(attention output of a 70B-shaped layer, three sequence lengths)")
     ap.add_argument("--comm-curve", action="store_true",
                     help="consumer bandwidth in isolation against the number of consumer CTAs (App. A)")
     ap.add_argument("--comm-ctas", type=int, default=0,
@@ -454,6 +524,8 @@ def main():
         return run_sweep(args, peaks, flush, torch, E, I)
     if args.ablation:
         return run_ablation(args, peaks, flush, torch, E, I)
+    if args.layer_chain:
+        return run_layer_chain(args, peaks, flush, torch, E, I)
     if args.comm_curve:
         # every input available, no competing producer: bandwidth against the budget (App. A)
         A, Bm = I.make_operands(wl, device="cuda")

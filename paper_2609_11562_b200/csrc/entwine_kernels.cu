@@ -133,6 +133,7 @@ struct KMaps {
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
   CUtensorMap p_ld[2];      // incoming partials as a 3-D tensor [W-1][M][N], box 128 x rs x (W-1):
                             // one load brings all peers' rows of a reduce step
+  CUtensorMap res_ld[2];    // layer chain: residual [R, N], box 128 x prs (a tile's residual, ahead of its reduce steps)
   CUtensorMap c_push[2];    // partial C, box 128 x prs: one load per push step
   CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N], box 128 x prs: one store per push step
   CUtensorMap p_pf;         // incoming partials, whole-tile box, for L2 prefetch
@@ -435,7 +436,8 @@ __device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) 
 // status helpers
 // ------------------------------------------------------------------------------------------
 struct SlotMeta {
-  int kind;      // 0 reduce step, 1 push step, 2 normalisation of a tile, -1 end of work, -2 continue on ring B
+  int kind;      // 0 reduce step, 1 push step, 2 normalisation of a tile, 3 residual rows of the tile whose
+                 // reduce steps follow, -1 end of work, -2 continue on ring B
   int dst_x;     // column of the destination box
   int dst_y;     // row of the destination box in the destination buffer
   int aux;       // layer chain: band (tile row) whose count the last step of a reduce task raises, else -1
@@ -557,6 +559,165 @@ __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KPar
   return r;
 }
 
+// The reducing warps' loop (Sec. 4.2, ReduceTile).  NORM selects the layer-chain variant, which
+// carries the tile's residual in registers and handles the residual and normalisation steps; the
+// plain variant is compiled without any of that state.
+template <bool NORM>
+__device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, uint32_t smem_base, Ring ring) {
+  const int lane = threadIdx.x & 31;
+  const int ctid = threadIdx.x - kRedWarp0 * 32;
+  int slot = -1;
+  uint32_t ph = 0;
+  // layer chain: this thread's 8 chunks (16 bytes each) of the residual of the tile being
+  // reduced: chunks ctid, ctid + 256, ... of the tile's 128 rows x 16 chunks
+  constexpr int kResChunks = kTile * (kTile * 2 / 16) / kRedThreads;
+  uint4 resv[kResChunks];
+#pragma unroll
+  for (int k = 0; k < kResChunks; ++k) resv[k] = make_uint4(0u, 0u, 0u, 0u);
+  for (;;) {
+    if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
+    // one lane per warp polls; the warp-level vote carries the barrier's acquire to all lanes
+    bool landed = true;
+    if (lane == 0) landed = mbar_wait(ring.full(slot), ph, P, sh);
+    if (!__all_sync(0xffffffffu, landed)) {
+      sh->abort = 1;
+      break;
+    }
+    const SlotMeta m = sh->meta[ring.id][slot];
+    if (m.kind == -1) break;
+    if (m.kind == -2) {
+      ring = make_ring(smem_base, 1, P);
+      slot = -1;
+      ph = 0;
+      continue;
+    }
+    if (!NORM && m.kind == 0) {
+      const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+      const int rs = ring.rs, sub_bytes = ring.sub_bytes;
+      __nv_bfloat16* dst = P.out + (long long)m.dst_y * P.N + m.dst_x;
+      // start from the local contribution, add the peers in ascending rank order, fp32; every
+      // thread writes its own 16 bytes of the output (single writer, 256-byte row segments)
+      for (int c = ctid; c < rs * (kTile * 2 / 16); c += kRedThreads) {
+        float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        const uint32_t addr = sbase + c * 16;
+        acc_bf16x8(a, ld_shared_v4(addr));
+#pragma unroll 4
+        for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
+        __stcs(reinterpret_cast<uint4*>(dst + (long long)(c >> 4) * P.N + (c & 15) * 8), pack_bf16x8(a));
+      }
+    } else if (NORM && m.kind == 0) {
+      // Layer chain (Sec. 5.2.3): the same rank-order fp32 sum, plus the residual; the bf16
+      // result is the new residual stream (written to P.out), and the sum of squares of the
+      // 128 stored values of each row inside this tile goes to ssq_part (one writer each).
+      const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+      const int rs = ring.rs, sub_bytes = ring.sub_bytes;
+      const int n_chunks = rs * (kTile * 2 / 16);
+      for (int c0 = 0; c0 < n_chunks; c0 += kRedThreads) {
+        const int c = c0 + ctid;
+        const bool act = c < n_chunks;
+        float ssq = 0.f;
+        if (act) {
+          const long long off = (long long)(m.dst_y + (c >> 4)) * P.N + m.dst_x + (c & 15) * 8;
+          float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          const uint32_t addr = sbase + c * 16;
+          acc_bf16x8(a, ld_shared_v4(addr));
+#pragma unroll 4
+          for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
+          // the residual, last: chunk (row of the tile) * 16 + (c & 15) of the tile, kept by this
+          // thread (or, for steps of fewer than 16 rows, read from global memory)
+          const int g = ((m.dst_y & (kTile - 1)) * (kTile * 2 / 16) + c) / kRedThreads;
+          uint4 rv = make_uint4(0u, 0u, 0u, 0u);
+          if (rs * (kTile * 2 / 16) >= kRedThreads) {
+#pragma unroll
+            for (int k = 0; k < kResChunks; ++k)
+              if (k == g) rv = resv[k];
+          } else {
+            rv = __ldcs(reinterpret_cast<const uint4*>(P.residual + off));
+          }
+          acc_bf16x8(a, rv);
+          const uint4 o = pack_bf16x8(a);
+          __stcg(reinterpret_cast<uint4*>(P.out + off), o);  // re-read from L2 by the normalisation
+          float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          acc_bf16x8(h, o);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) ssq = fmaf(h[e], h[e], ssq);
+        }
+        // the 16 threads of a row segment (half a warp) add up in a fixed order
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
+        if (act && (lane & 15) == 0)
+          __stcg(&P.ssq_part[(long long)(m.dst_y + (c >> 4)) * P.nTn + m.dst_x / kTile], ssq);
+      }
+    } else if (NORM && m.kind == 3) {
+      // residual rows [dst_y, dst_y + prs) of the tile: every thread takes its chunks
+      const uint32_t sbase = ring.base + slot * ring.slot_bytes;
+      const int g0 = m.dst_y * (kTile * 2 / 16), g1 = g0 + ring.prs * (kTile * 2 / 16);
+#pragma unroll
+      for (int k = 0; k < kResChunks; ++k) {
+        const int g = ctid + k * kRedThreads;
+        if (g >= g0 && g < g1) resv[k] = ld_shared_v4(sbase + (g - g0) * 16);
+      }
+    } else if (NORM && m.kind == 2) {
+      // Normalisation of one 128 x 128 tile of a complete band: 1/RMS of each of its rows from
+      // the nTn partial sums (fixed order), then hidden * inv_rms * weight, rounded once.
+      // two threads per row: each adds its half of the row's nTn partial sums (all loads in
+      // flight together where the halves are 16-byte aligned), one shuffle joins the halves;
+      // the order of the additions is fixed
+      {
+        const int row = ctid >> 1, half = ctid & 1;
+        const int n_half = (P.nTn + 1) / 2;
+        const int first = half * n_half;
+        const int cnt = min(n_half, P.nTn - first);
+        const float* pr = P.ssq_part + (long long)(m.dst_y + row) * P.nTn + first;
+        float sum = 0.f;
+        if ((P.nTn & 7) == 0) {
+          for (int q0 = 0; q0 < cnt; q0 += 32) {
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              v[j] = (q0 + 4 * j < cnt) ? __ldcg(reinterpret_cast<const float4*>(pr + q0 + 4 * j))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sum += (v[j].x + v[j].y) + (v[j].z + v[j].w);
+          }
+        } else {
+          for (int q = 0; q < cnt; ++q) sum += __ldcg(pr + q);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        if (half == 0) sh->inv_rms[row] = rsqrtf(sum / (float)P.N + P.eps);
+      }
+      named_bar_sync(2, kRedThreads);
+      float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      acc_bf16x8(w, __ldg(reinterpret_cast<const uint4*>(P.weight + m.dst_x + (ctid & 15) * 8)));
+      // 8 independent 16-byte loads per thread in flight, then the arithmetic and the stores
+      constexpr int kIter = kTile * (kTile * 2 / 16) / kRedThreads;
+      uint4 hv[kIter];
+#pragma unroll
+      for (int k = 0; k < kIter; ++k) {
+        const int c = ctid + k * kRedThreads;
+        hv[k] = __ldcg(reinterpret_cast<const uint4*>(P.out + (long long)(m.dst_y + (c >> 4)) * P.N + m.dst_x + (c & 15) * 8));
+      }
+#pragma unroll
+      for (int k = 0; k < kIter; ++k) {
+        const int c = ctid + k * kRedThreads;
+        const int row = c >> 4;
+        float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        acc_bf16x8(h, hv[k]);
+        const float inv = sh->inv_rms[row];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) h[e] = h[e] * inv * w[e];
+        __stcs(reinterpret_cast<uint4*>(P.norm_out + (long long)(m.dst_y + row) * P.N + m.dst_x + (c & 15) * 8),
+               pack_bf16x8(h));
+      }
+      named_bar_sync(2, kRedThreads);  // inv_rms is rewritten by the next normalisation step
+    }
+    // one arrival per warp returns the slot (a push step is forwarded by the store warp alone;
+    // the arrival then only says that this warp has read the slot's header)
+    __syncwarp();
+    if (lane == 0) mbar_arrive(ring.red(slot));
+  }
+}
+
 // One CTA's consumer work, run by warps 2, 3 and 8-15.  Warp 2 claims tasks from `n_lists`
 // consumer lists starting at `first_list` (each list is consumed in order through its head
 // counter, Sec. 3.1), polls the tile flags with one lane per contributing rank, and streams
@@ -564,7 +725,8 @@ __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KPar
 // and write the result; warp 3 forwards pushed tiles with TMA stores and recycles the slots.
 // In a producer CTA the pipeline starts on the small ring A beside the producer's buffers and
 // moves to ring B (the producer's buffers) once `gemm_done` is set.
-__device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
+template <bool NORM>
+__device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
                                   int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P);
@@ -756,14 +918,30 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
             int slot = it % ring.n_slots;
             uint32_t ph = (it / ring.n_slots) & 1;
             const uint32_t tx = kind == 0 ? P.W * ring.sub_bytes : ring.prs * kTile * 2;
-            for (int step = 0; step < n_steps; ++step) {
+            if (NORM && kind == 0) {
+              // layer chain: the tile's residual rows first (whole push-sized steps); the reducing
+              // warps keep them in registers for the reduce steps that follow
+              for (int u = 0; u < kTile / ring.prs; ++u) {
+                if (!mbar_wait(ring.empty(slot), ph ^ 1, P, sh)) { steps_ok = false; break; }
+                SlotMeta& m = sh->meta[ring.id][slot];
+                m.kind = 3;
+                m.dst_x = col;
+                m.dst_y = u * ring.prs;  // first row of these residual rows inside the tile
+                m.aux = -1;
+                mbar_arrive_expect_tx(ring.full(slot), ring.prs * kTile * 2);
+                tma_load_2d_hint(ring.base + slot * ring.slot_bytes, &maps.res_ld[ring.geom], col,
+                                 dst_row + u * ring.prs, ring.full(slot), pol);
+                if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
+              }
+            }
+            for (int step = 0; steps_ok && step < n_steps; ++step) {
               if (!mbar_wait(ring.empty(slot), ph ^ 1, P, sh)) { steps_ok = false; break; }
               const uint32_t dst = ring.base + slot * ring.slot_bytes;
               SlotMeta& m = sh->meta[ring.id][slot];
               m.kind = kind;
               m.dst_x = col;
               m.dst_y = dst_row + step * rows;
-              m.aux = (P.norm && kind == 0 && step == n_steps - 1) ? dst_row / kTile : -1;
+              m.aux = (NORM && kind == 0 && step == n_steps - 1) ? dst_row / kTile : -1;
               mbar_arrive_expect_tx(ring.full(slot), tx);
               // Few, large TMA operations: the per-operation cost of the TMA unit, not bandwidth,
               // bounds a consumer that issues many small boxes.
@@ -773,6 +951,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
                 tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
                 tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
                                  ring.full(slot), pol);
+
               } else {
                 tma_load_2d_hint(dst, &maps.c_push[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
               }
@@ -786,7 +965,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
             }
           }
           ok = __all_sync(0xffffffffu, steps_ok);
-          it += n_steps;
+          it += n_steps + ((NORM && kind == 0) ? kTile / ring.prs : 0);
         }
       }
     };
@@ -817,26 +996,34 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
     // tasks (one per tile of the rank's partition, band by band) through one counter.  A task
     // waits until all nTn tiles of its band are reduced; the reducing warps read the band from
     // L2 themselves, the ring slot only hands them the task.
-    if (P.norm && ok && n_lists > 0) {
+    if (NORM && ok && n_lists > 0) {
       int* head = &P.list_head[P.x];
-      int c0 = P.Q, c1 = P.Q;
-      if (lane == 0) {
-        c0 = atomicAdd(head, 1);
-        c1 = atomicAdd(head, 1);
-      }
       while (ok) {
-        const int i = __shfl_sync(0xffffffffu, c0, 0);
-        if (i >= P.Q) break;
-        c0 = c1;
-        if (lane == 0) c1 = atomicAdd(head, 1);
-        const int band = i / P.nTn, tc = i - band * P.nTn;
+        // Wait for the band at the head of the task counter BEFORE claiming: a CTA that waits
+        // holds no task, so the tasks of a band that completes are shared by every CTA that is
+        // free at that moment.
+        int i = P.Q;
         bool band_ok = true;
-        if (lane == 0) band_ok = wait_count(&P.band_ctr[band], (unsigned)P.nTn, P);
+        if (lane == 0) {
+          const int peek = *reinterpret_cast<volatile int*>(head);
+          if (peek < P.Q) {
+            band_ok = wait_count(&P.band_ctr[peek / P.nTn], (unsigned)P.nTn, P);
+            if (band_ok) {
+              i = atomicAdd(head, 1);
+              // the claim may belong to the next band already
+              if (i < P.Q && i / P.nTn != peek / P.nTn)
+                band_ok = wait_count(&P.band_ctr[i / P.nTn], (unsigned)P.nTn, P);
+            }
+          }
+        }
         ok = __all_sync(0xffffffffu, band_ok);
         if (!ok) {
           if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, -7);
           break;
         }
+        i = __shfl_sync(0xffffffffu, i, 0);
+        if (i >= P.Q) break;
+        const int band = i / P.nTn, tc = i - band * P.nTn;
         maybe_switch();
         if (!ok) break;
         bool free_slot = true;
@@ -867,103 +1054,7 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
     __syncwarp();
   } else if (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32) {
     // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
-    const int ctid = threadIdx.x - kRedWarp0 * 32;
-    int slot = -1;
-    uint32_t ph = 0;
-    for (;;) {
-      if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
-      // one lane per warp polls; the warp-level vote carries the barrier's acquire to all lanes
-      bool landed = true;
-      if (lane == 0) landed = mbar_wait(ring.full(slot), ph, P, sh);
-      if (!__all_sync(0xffffffffu, landed)) {
-        sh->abort = 1;
-        break;
-      }
-      const SlotMeta m = sh->meta[ring.id][slot];
-      if (m.kind == -1) break;
-      if (m.kind == -2) {
-        ring = make_ring(smem_base, 1, P);
-        slot = -1;
-        ph = 0;
-        continue;
-      }
-      if (m.kind == 0 && !P.norm) {
-        const uint32_t sbase = ring.base + slot * ring.slot_bytes;
-        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
-        __nv_bfloat16* dst = P.out + (long long)m.dst_y * P.N + m.dst_x;
-        // start from the local contribution, add the peers in ascending rank order, fp32; every
-        // thread writes its own 16 bytes of the output (single writer, 256-byte row segments)
-        for (int c = ctid; c < rs * (kTile * 2 / 16); c += kRedThreads) {
-          float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          const uint32_t addr = sbase + c * 16;
-          acc_bf16x8(a, ld_shared_v4(addr));
-#pragma unroll 4
-          for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
-          __stcs(reinterpret_cast<uint4*>(dst + (long long)(c >> 4) * P.N + (c & 15) * 8), pack_bf16x8(a));
-        }
-      } else if (m.kind == 0) {
-        // Layer chain (Sec. 5.2.3): the same rank-order fp32 sum, plus the residual; the bf16
-        // result is the new residual stream (written to P.out), and the sum of squares of the
-        // 128 stored values of each row inside this tile goes to ssq_part (one writer each).
-        const uint32_t sbase = ring.base + slot * ring.slot_bytes;
-        const int rs = ring.rs, sub_bytes = ring.sub_bytes;
-        const int n_chunks = rs * (kTile * 2 / 16);
-        for (int c0 = 0; c0 < n_chunks; c0 += kRedThreads) {
-          const int c = c0 + ctid;
-          const bool act = c < n_chunks;
-          float ssq = 0.f;
-          if (act) {
-            const long long off = (long long)(m.dst_y + (c >> 4)) * P.N + m.dst_x + (c & 15) * 8;
-            const uint4 res = __ldcs(reinterpret_cast<const uint4*>(P.residual + off));
-            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            const uint32_t addr = sbase + c * 16;
-            acc_bf16x8(a, ld_shared_v4(addr));
-#pragma unroll 4
-            for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_shared_v4(addr + q * sub_bytes));
-            acc_bf16x8(a, res);
-            const uint4 o = pack_bf16x8(a);
-            __stcg(reinterpret_cast<uint4*>(P.out + off), o);  // re-read from L2 by the normalisation
-            float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            acc_bf16x8(h, o);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) ssq = fmaf(h[e], h[e], ssq);
-          }
-          // the 16 threads of a row segment (half a warp) add up in a fixed order
-#pragma unroll
-          for (int o = 8; o > 0; o >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, o);
-          if (act && (lane & 15) == 0)
-            __stcg(&P.ssq_part[(long long)(m.dst_y + (c >> 4)) * P.nTn + m.dst_x / kTile], ssq);
-        }
-      } else if (m.kind == 2) {
-        // Normalisation of one 128 x 128 tile of a complete band: 1/RMS of each of its rows from
-        // the nTn partial sums (fixed order), then hidden * inv_rms * weight, rounded once.
-        if (ctid < kTile) {
-          const float* pr = P.ssq_part + (long long)(m.dst_y + ctid) * P.nTn;
-          float sum = 0.f;
-          for (int tc = 0; tc < P.nTn; ++tc) sum += __ldcg(pr + tc);
-          sh->inv_rms[ctid] = rsqrtf(sum / (float)P.N + P.eps);
-        }
-        named_bar_sync(2, kRedThreads);
-        float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        acc_bf16x8(w, __ldg(reinterpret_cast<const uint4*>(P.weight + m.dst_x + (ctid & 15) * 8)));
-#pragma unroll 4
-        for (int c = ctid; c < kTile * (kTile * 2 / 16); c += kRedThreads) {
-          const int row = c >> 4;
-          const long long off = (long long)(m.dst_y + row) * P.N + m.dst_x + (c & 15) * 8;
-          float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          acc_bf16x8(h, __ldcg(reinterpret_cast<const uint4*>(P.out + off)));
-          const float inv = sh->inv_rms[row];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) h[e] = h[e] * inv * w[e];
-          __stcs(reinterpret_cast<uint4*>(P.norm_out + off), pack_bf16x8(h));
-        }
-        named_bar_sync(2, kRedThreads);  // inv_rms is rewritten by the next normalisation step
-      }
-      // one arrival per warp returns the slot (a push step is forwarded by the store warp alone;
-      // the arrival then only says that this warp has read the slot's header)
-      __syncwarp();
-      if (lane == 0) mbar_arrive(ring.red(slot));
-    }
+    reducer_role<NORM>(P, sh, smem_base, ring);
   } else if (warp == kStoreWarp && lane == 0) {
     // ---------------- forward push slots with TMA stores, recycle all slots ----------------
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
@@ -1006,8 +1097,8 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
         sh->abort = 1;
         break;
       }
-      if (m.kind == 0 || m.kind == 2) {
-        if (m.aux >= 0) {
+      if (m.kind == 0 || (NORM && (m.kind == 2 || m.kind == 3))) {
+        if (NORM && m.aux >= 0) {
           // layer chain: the last step of a reduce task counts its tile in the band
           fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
           atomicAdd(&P.band_ctr[m.aux], 1u);
@@ -1034,7 +1125,9 @@ __device__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared
 // ------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------
-template <int BN, bool PAIR>
+// NORM: the layer-chain variant (residual add + RMSNorm in the consumer) is a kernel of its own,
+// so that the plain kernel's code and register allocation are untouched by it.
+template <int BN, bool PAIR, bool NORM>
 __global__ void __launch_bounds__(kThreads, 1)
 entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   using C = Cfg<BN, PAIR>;
@@ -1439,7 +1532,9 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         on_a = false;
       }
     }
-    if (count > 0 && !sh.abort) consumer_pipeline(P, maps, &sh, smem_base, first, count, on_a, &cnt);
+    if (count > 0 && !sh.abort) {
+      consumer_pipeline<NORM>(P, maps, &sh, smem_base, first, count, on_a, &cnt);
+    }
     if (warp == kCommWarp && lane == 0) {
       if (cnt.reduced) atomicAdd(&st->tiles_reduced, (unsigned long long)cnt.reduced);
       if (cnt.pushed) atomicAdd(&st->tiles_pushed, (unsigned long long)cnt.pushed);
@@ -1632,15 +1727,16 @@ void device_release(Plan* p) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-template <int BN, bool PAIR>
+template <int BN, bool PAIR, bool NORM = false>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
+  if (!NORM && kp.norm) return launch_bn<BN, PAIR, true>(p, kp, maps, grid, stream);
   // per device: the shared-memory opt-in has been set, and how many clusters fit at once
   static int max_clusters[64] = {0};
   static bool configured[64] = {false};
   int dev = 0;
   CK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ENTWINE_ERR_RESOURCES;
-  auto kern = entwine_fused_kernel<BN, PAIR>;
+  auto kern = entwine_fused_kernel<BN, PAIR, NORM>;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(unsigned(grid), 1, 1);
@@ -1674,14 +1770,18 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
 // contributions (at most 16 KiB with geometry 0, 32 KiB with geometry 1), a push step moves as
 // many rows of one tile as fit in a slot.  The producer's operand ring gets `stages` stages;
 // what remains after the epilogue staging is the co-located consumer ring A.
-static int ring_geometry(const Plan* p, KParams* kp) {
+// `extra` = contributions a reduce step carries besides the W partial outputs (the residual of the
+// layer chain).
+static int ring_geometry(const Plan* p, KParams* kp, int extra = 0) {
   const Geometry& g = p->g;
   for (int id = 0; id < 2; ++id) {
     const int budget = id == 0 ? 16384 : 32768;
     int rs = 1;
-    while (int64_t(g.W) * (rs * 2) * kTile * 2 <= budget && rs * 2 <= kTile) rs *= 2;
-    int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
-    slot_bytes = (slot_bytes + 1023) / 1024 * 1024;
+    while (int64_t(g.W + extra) * (rs * 2) * kTile * 2 <= budget && rs * 2 <= kTile) rs *= 2;
+    // a slot is as large as the budget even when a reduce step fills less of it (W + extra not a
+    // power of two): push steps, most of the traffic, then keep their full size
+    int slot_bytes = int(int64_t(g.W + extra) * rs * kTile * 2);
+    slot_bytes = std::max((slot_bytes + 1023) / 1024 * 1024, budget);
     int prs = rs;
     while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
     kp->rs[id] = rs;
@@ -1863,7 +1963,8 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
          make_map(&maps.c_push[id], c_src, g.M, g.N, kTile, prs, false) &&
          (comm ? make_map3(&maps.p_ld[id], peers, g.W - 1, g.M, g.N, kTile, rs, g.W - 1)
                : make_map3(&maps.p_ld[id], d->C, 1, g.M, g.N, kTile, rs, 1)) &&
-         make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, prs, false);
+         make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, prs, false) &&
+         make_map(&maps.res_ld[id], norm ? norm->residual : d->C, norm ? g.R : g.M, g.N, kTile, prs, false);
   }
   if (!ok) return ENTWINE_ERR_CUDA;
   if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
