@@ -1798,6 +1798,8 @@ static int ring_geometry(const Plan* p, KParams* kp, int extra = 0) {
     const double t_tc = 2.0 * g.M * g.N * g.K / 1.6e15;
     const double t_hbm = double(g.M) * g.N * 2.0 * (3 * g.W - 1) / g.W / 6.5e12;
     if (p->colocate && t_hbm > 0.5 * t_tc && stages > 3) stages -= 1;
+    // communication-bound shapes (K_local of a few hundred): one more stage goes to the ring
+    if (p->colocate && t_hbm > t_tc && stages > 3) stages -= 1;
   }
   if (stages < 2 || stages > kMaxStages) return ENTWINE_ERR_INVALID;
   const int ring_a_off = stages * stage_bytes + kStagingBytes;
