@@ -875,10 +875,11 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
             continue;
           }
-          if (P.prefetch && c + 1 < n) {
-            // Look-ahead: if the next task of the claim is a reduce task whose peer contributions
-            // are already published, pull their tiles into L2 now (one lane per peer) so that the
-            // ring's loads find them there while holding a slot.
+          if (P.prefetch && i + 1 < len && src + 1 < 32) {
+            // Look-ahead: if the list's next task is a reduce task whose peer contributions are
+            // already published, pull their tiles into L2 now (one lane per peer) so that the
+            // ring's loads find them there while holding a slot.  (The task may end up with
+            // another CTA; the tiles are in L2 for it all the same.)
             const int nkind = __shfl_sync(0xffffffffu, k_kind, src + 1);
             const int nt = __shfl_sync(0xffffffffu, k_t, src + 1);
             const int nrow = __shfl_sync(0xffffffffu, k_row, src + 1);
