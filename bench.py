@@ -679,7 +679,7 @@ def main():
         names = [wl.name] + [n for n in ("attn_out_proj", "mlp_down_proj", "short_k_comm_bound") if n != wl.name]
         for name in names:
             w2 = I.CONFIGS[name]
-            r = measure_workload(w2, LAUNCH[name], max(10, args.steps // 2), 5, flush, torch, E, I, True)
+            r = measure_workload(w2, LAUNCH[name], min(100, max(10, args.steps // 2)), 5, flush, torch, E, I, True)
             med = statistics.median
             fused = med(r["fused_us"])
             tc, hb = roofline_seconds(w2, peaks)
@@ -701,7 +701,7 @@ def main():
                 "tile_order": "interleaved" if LAUNCH[name]["order"] else "row_major",
             }
             other = dict(LAUNCH[name], order=1 - LAUNCH[name]["order"])
-            r2 = measure_workload(w2, other, max(10, args.steps // 2), 5, flush, torch, E, I, False)
+            r2 = measure_workload(w2, other, min(100, max(10, args.steps // 2)), 5, flush, torch, E, I, False)
             e["other_tile_order_fused_us"] = med(r2["fused_us"])
             # Eq. 4 generalised to the emulation's push + reduce bytes, from the measured window
             t_g = r["status"]["t_gemm_ns"] * 1e-9
