@@ -782,10 +782,17 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       const int len = P.list_offs[j + 1] - base;
       if (len <= 0) return;
       const int CH = P.claim;  // CH * W <= 64 (W <= 64): the flags of a claim fit the early look
-      // Claims shrink towards the end of the list (guided self-scheduling) so that the CTAs that
-      // share it finish together: a quarter of an even share of what is left, at most CH tasks.
+      // Where several CTAs share a list, claims shrink towards its end (guided self-scheduling)
+      // so that they finish together: a quarter of an even share of what is left, at most CH
+      // tasks.  A list with one CTA of its own is claimed CH tasks at a time to the end: the
+      // fence that turns a claim's early flag reads into an acquire waits for the claim atomic in
+      // flight, and is paid once per claim.
       const int sharers = ((int)gridDim.x + P.x - 1) / P.x;
-      auto claim_len = [&](int head) { return max(1, min(CH, (len - head) / (4 * sharers))); };
+      auto claim_len = [&](int head) {
+        // (longer claims on shared lists measured slower: the tiles in flight at one time then
+        // lie further apart in memory)
+        return sharers > 1 ? max(1, min(min(CH, 2), (len - head) / (4 * sharers))) : max(1, min(CH, len - head));
+      };
       int cur = len, nxt = len, fut = len;
       int cur_n = claim_len(0), nxt_n = cur_n, fut_n = cur_n;
       if (lane == 0) {
@@ -1623,10 +1630,9 @@ static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_
 }
 
 // Tasks per claim: as many as have their flags (W per reduce task) in the 64 flag values the
-// claiming warp reads ahead, at most two.  Longer claims measured slower where several CTAs
-// share a list: the tiles in flight at one time then lie further apart in memory.
+// claiming warp reads ahead, at most four (two where several CTAs share a list).
 #ifndef ENTWINE_CLAIM_MAX
-#define ENTWINE_CLAIM_MAX 2
+#define ENTWINE_CLAIM_MAX 4
 #endif
 static int claim_size(int W) { return std::max(1, std::min(ENTWINE_CLAIM_MAX, 64 / W)); }
 
