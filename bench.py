@@ -650,6 +650,10 @@ def main():
         achieved = wl.comm_bytes / (mean_us * 1e-6) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"]}
+    # the same time against the other denominators: the seconds-long cuBLAS figure under the power
+    # cap, and the nominal HBM bandwidth
+    t_alt = max(wl.flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12), wl.comm_bytes / 8.0e12)
+    roof["frac_vs_sustained_tensor_and_nominal_hbm"] = t_alt / (mean_us * 1e-6)
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
     roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
