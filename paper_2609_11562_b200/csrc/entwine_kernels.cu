@@ -1777,17 +1777,15 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
 // contributions (at most 16 KiB with geometry 0, 32 KiB with geometry 1), a push step moves as
 // many rows of one tile as fit in a slot.  The producer's operand ring gets `stages` stages;
 // what remains after the epilogue staging is the co-located consumer ring A.
-// `extra` = contributions a reduce step carries besides the W partial outputs (the residual of the
-// layer chain).
-static int ring_geometry(const Plan* p, KParams* kp, int extra = 0) {
+static int ring_geometry(const Plan* p, KParams* kp) {
   const Geometry& g = p->g;
   for (int id = 0; id < 2; ++id) {
     const int budget = id == 0 ? 16384 : 32768;
     int rs = 1;
-    while (int64_t(g.W + extra) * (rs * 2) * kTile * 2 <= budget && rs * 2 <= kTile) rs *= 2;
-    // a slot is as large as the budget even when a reduce step fills less of it (W + extra not a
+    while (int64_t(g.W) * (rs * 2) * kTile * 2 <= budget && rs * 2 <= kTile) rs *= 2;
+    // a slot is as large as the budget even when a reduce step fills less of it (W not a
     // power of two): push steps, most of the traffic, then keep their full size
-    int slot_bytes = int(int64_t(g.W + extra) * rs * kTile * 2);
+    int slot_bytes = int(int64_t(g.W) * rs * kTile * 2);
     slot_bytes = std::max((slot_bytes + 1023) / 1024 * 1024, budget);
     int prs = rs;
     while (prs < kTile && int64_t(prs) * 2 * kTile * 2 <= slot_bytes) prs *= 2;
