@@ -719,7 +719,7 @@ def main():
     if not args.no_cpu_baseline:
         rows = wl.M if wl.flops <= 5e10 else 512
         probe, _, _ = run_cpu_oracle(wl, launch, rows, 1)
-        passes = int(max(3, min(40, 12.0 / max(probe[0], 1e-3))))
+        passes = int(max(3, min(80, 15.0 / max(probe[0], 1e-3))))  # about 15 s of CPU work
         times, flops, threads = run_cpu_oracle(wl, launch, rows, passes)
         line["cpu_baseline"] = {
             "value": flops / min(times) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
