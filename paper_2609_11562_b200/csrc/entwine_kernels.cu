@@ -92,6 +92,9 @@ struct KParams {
   int l2_hints;   // consumer TMA traffic carries an evict-first L2 policy
   int stages;     // operand-ring stages of the producer
   int ring_a_off, ring_a_bytes;  // consumer ring A (after the epilogue staging)
+  int stage_area;                // bytes of the operand stages
+  int early_b;                   // 1: a producer CTA's ring B is its operand stages, used as soon as its
+                                 // last MMA has completed; 0: the full ring B once its producer work is over
   int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
   int skip_wait;  // treat every flag as published (consumer in isolation)
   int claim;      // most consecutive tasks taken from a list per claim
@@ -445,6 +448,9 @@ struct SlotMeta {
 struct CtaShared {
   volatile int abort;      // a role of this CTA (or another CTA) gave up
   volatile int gemm_done;  // this CTA's producer work is over; its shared memory is free
+  volatile int stages_free;  // the CTA's last MMA has completed: its operand stages are free
+  int ring_b_bytes;          // size of this CTA's ring B: the operand stages of a producer CTA (ring B
+                             // then starts before the epilogue is over), 192 KiB of a consumer CTA
   int blocks_stored;       // blocks of this CTA whose partial-C stores are complete
   float inv_rms[kTile];    // layer chain: 1 / RMS of the rows of the tile being normalised
   SlotMeta meta[2][kMaxSlots];
@@ -545,7 +551,7 @@ struct Ring {
   __device__ __forceinline__ uint32_t empty(int s) const { return bars + 8u * (kMaxSlots + s); }
   __device__ __forceinline__ uint32_t red(int s) const { return bars + 8u * (2 * kMaxSlots + s); }
 };
-__device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KParams& P) {
+__device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KParams& P, const CtaShared* sh) {
   Ring r;
   r.id = id;
   r.geom = id == 0 ? P.ring_a_geom : 1;
@@ -555,7 +561,7 @@ __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KPar
   r.prs = P.prs[r.geom];
   r.slot_bytes = P.slot_bytes[r.geom];
   r.sub_bytes = r.rs * kTile * 2;
-  r.n_slots = min(kMaxSlots, (id == 0 ? P.ring_a_bytes : kRingBBytes) / r.slot_bytes);
+  r.n_slots = min(kMaxSlots, (id == 0 ? P.ring_a_bytes : sh->ring_b_bytes) / r.slot_bytes);
   return r;
 }
 
@@ -586,7 +592,7 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
     const SlotMeta m = sh->meta[ring.id][slot];
     if (m.kind == -1) break;
     if (m.kind == -2) {
-      ring = make_ring(smem_base, 1, P);
+      ring = make_ring(smem_base, 1, P, sh);
       slot = -1;
       ph = 0;
       continue;
@@ -729,7 +735,7 @@ template <bool NORM>
 __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
                                   int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P);
+  Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P, sh);
 
   if (warp == kCommWarp) {
     // ---------------- claim, poll, load ----------------
@@ -742,27 +748,30 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     auto maybe_switch = [&]() {
       if (ring.id != 0) return;
       int done = 0;
-      if (lane == 0) done = sh->gemm_done;
+      if (lane == 0) done = P.early_b ? sh->stages_free : sh->gemm_done;
       done = __shfl_sync(0xffffffffu, done, 0);
       if (!done) return;
       bool free_slot = true;
       if (lane == 0) {
-        // Ring B overlaps ring A's memory: every step still in flight in ring A must have been
-        // reduced or forwarded (its slot returned) before ring B is loaded.  Slot s has been
-        // used uses(s) times; its last use, number uses(s) - 1, is over when the empty barrier
-        // completes the phase of that parity.
-        for (int sl = 0; free_slot && sl < ring.n_slots; ++sl) {
+        // With early_b, ring B lies in the operand stages only, which neither ring A nor the
+        // epilogue's staging overlaps: steps still in flight in ring A are not disturbed.
+        // Otherwise ring B's last slots overlap ring A's memory, and every ring-A step in flight
+        // must have returned its slot first: slot s has been used uses(s) times; its last use,
+        // number uses(s) - 1, is over when its empty barrier completes the phase of that parity.
+        for (int sl = 0; !P.early_b && free_slot && sl < ring.n_slots; ++sl) {
           const int uses = (it - sl + ring.n_slots - 1) / ring.n_slots;
           if (uses > 0) free_slot = mbar_wait(ring.empty(sl), (uses - 1) & 1, P, sh);
         }
+        // the marker travels through the next ring-A slot, which must be free
+        const int slot = it % ring.n_slots;
+        if (free_slot) free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
         if (free_slot) {
-          const int slot = it % ring.n_slots;
           sh->meta[0][slot].kind = -2;
           mbar_arrive(ring.full(slot));
         }
       }
       ok = __all_sync(0xffffffffu, free_slot);
-      ring = make_ring(smem_base, 1, P);
+      ring = make_ring(smem_base, 1, P, sh);
       it = 0;
     };
     // Drains list j.  Claims go through the list's head counter in runs of up to P.claim
@@ -1076,7 +1085,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       if (!n_pend) return;
       bulk_wait_read<0>();
       for (; n_pend > 0; --n_pend, pend >>= 8) {
-        const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P);
+        const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P, sh);
         mbar_arrive(rr.empty(int(pend & 15u)));
       }
     };
@@ -1095,7 +1104,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       if (m.kind == -1) break;
       if (m.kind == -2) {
         retire_all();
-        ring = make_ring(smem_base, 1, P);
+        ring = make_ring(smem_base, 1, P, sh);
         slot = -1;
         ph = 0;
         continue;
@@ -1117,7 +1126,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
-          const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P);
+          const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P, sh);
           mbar_arrive(rr.empty(int(pend & 15u)));
           pend >>= 8;
           --n_pend;
@@ -1186,6 +1195,8 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     sh.abort = 0;
     sh.blocks_stored = 0;
     sh.gemm_done = (is_producer && n_my > 0) ? 0 : 1;
+    sh.stages_free = (is_producer && n_my > 0) ? 0 : 1;
+    sh.ring_b_bytes = (is_producer && n_my > 0 && P.early_b) ? P.stage_area : kRingBBytes;
     atomicMin(&st->t_start, globaltimer_ns());
     if (is_producer) {
       for (int s = 0; s < n_stages; ++s) {
@@ -1321,6 +1332,11 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         ok = __all_sync(0xffffffffu, ok);  // reconverge; the warp leaves the loop together
         if (!ok) break;
         tc_fence_after();
+        if (i == n_my - 1 && warp == kEpiWarp0 && lane == 0) {
+          // the CTA's (and, on a pair, the cluster's) last MMA has read the operand stages
+          __threadfence_block();
+          sh.stages_free = 1;
+        }
         const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + acc * BN;
 #pragma unroll 1
         for (int j = 0; j < BN / 64; ++j, ++nbox) {
@@ -1533,7 +1549,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       if (count > 0 && on_a && !P.colocate) {
         // not co-located: wait for the CTA's producer work to end, then use ring B
         unsigned long long t0 = globaltimer_ns();
-        while (!sh.gemm_done && !sh.abort) {
+        while (!(P.early_b ? sh.stages_free : sh.gemm_done) && !sh.abort) {
           __nanosleep(256);
           if (globaltimer_ns() - t0 > 64ULL * P.wait_budget_ns) break;
         }
@@ -1812,6 +1828,9 @@ static int ring_geometry(const Plan* p, KParams* kp) {
   if (ring_a_bytes < 2 * kp->slot_bytes[0]) return ENTWINE_ERR_RESOURCES;
   kp->stages = stages;
   kp->ring_a_off = ring_a_off;
+  kp->stage_area = std::min(stages * stage_bytes, kRingBBytes);
+  // ring B in the operand stages alone needs room for at least four slots to keep the tail's rate
+  kp->early_b = kp->stage_area >= 4 * kp->slot_bytes[1] ? 1 : 0;
   kp->ring_a_bytes = ring_a_bytes;
   kp->ring_a_geom = ring_a_bytes >= 2 * kp->slot_bytes[1] ? 1 : 0;
   return ENTWINE_OK;
