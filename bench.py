@@ -268,6 +268,7 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     res["fused_back_to_back_us"] = e0.elapsed_time(e1) * 1e3 / steps
     plan.last_status()
     if detailed:
+        time.sleep(0.5)  # the queued calls above are a sustained load: let the clock recover
         # the producer alone (uncontended GEMM time) and the consumer alone
         res["gemm_only_us"] = time_steps(lambda: plan.gemm_only(A, Bm), max(5, steps // 4), 3, flush, torch)
         plan.last_status()
@@ -682,6 +683,7 @@ def main():
         extra = {}
         names = [wl.name] + [n for n in ("attn_out_proj", "mlp_down_proj", "short_k_comm_bound") if n != wl.name]
         for name in names:
+            time.sleep(1.0)  # let the part recover from the previous workload's sustained load
             w2 = I.CONFIGS[name]
             r = measure_workload(w2, LAUNCH[name], min(100, max(10, args.steps // 2)), 5, flush, torch, E, I, True)
             med = statistics.median
