@@ -267,6 +267,32 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     torch.cuda.synchronize()
     res["fused_back_to_back_us"] = e0.elapsed_time(e1) * 1e3 / steps
     plan.last_status()
+    # CUDA-graph replay: the same queue of calls captured once (each preceded by the library's
+    # reset kernel, see include/entwine.h) and replayed between one event pair.  A plan of its
+    # own, so that the eager plan above keeps launching without the reset kernel.
+    n_cap = min(steps, 50)
+    gplan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=launch["rank"],
+                   **launch.get("opts", {}))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gplan.gemm_rs(A, Bm, P, out, send)
+        gplan.last_status()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(n_cap):
+                gplan.gemm_rs(A, Bm, P, out, send)
+        graph.replay()
+        side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        side.synchronize()
+        gplan.last_status()
+    res["fused_graph_replay_us"] = e0.elapsed_time(e1) * 1e3 / n_cap
+    del graph
+    gplan.destroy()
     if detailed:
         time.sleep(0.5)  # the queued calls above are a sustained load: let the clock recover
         # the producer alone (uncontended GEMM time) and the consumer alone
@@ -693,6 +719,7 @@ def main():
                 "fused_us": fused, "fused_tflops": w2.flops / fused / 1e6,
                 "fused_hot_l2_us": med(r["fused_hot_us"]),
                 "fused_back_to_back_us": r["fused_back_to_back_us"],
+                "fused_graph_replay_us": r["fused_graph_replay_us"],
                 "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
                 "bound": "tensor" if tc >= hb else "hbm",
                 "unfused_cublas_then_reduce_us": med(r["unfused_us"]),

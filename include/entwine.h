@@ -167,6 +167,14 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value);
  * ENTWINE_ERR_CUDA; a timeout or index failure of an earlier launch that
  * entwine_last_status has not yet collected is returned as ENTWINE_ERR_TIMEOUT /
  * ENTWINE_ERR_INTERNAL by that later query, never by a trap.
+ * CUDA graphs: entwine_gemm_rs, entwine_gemm_rs_norm, entwine_gemm_only and
+ * entwine_comm_only may be called on a capturing stream once the plan has made one launch of
+ * that kind outside a capture (the first launch allocates; a capture before it returns
+ * ENTWINE_ERR_INVALID).  A replay runs with the pointers and the flag value of the capture,
+ * so a captured call is preceded by a small kernel that clears the plan's flags, list heads
+ * and status, and so is every later call of that plan.  Replays of one plan must not overlap
+ * each other or its other launches; entwine_last_status after a replay reports that replay
+ * if the captured call was the plan's latest call.
  */
 int entwine_gemm_rs(entwine_plan_t plan, const void* A, const void* B,
                     const void* peer_partials, void* out_shard, void* send_bufs,

@@ -1140,6 +1140,29 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
 }
 
 // ------------------------------------------------------------------------------------------
+// Reset of a plan's launch state on the device.  A launch captured into a CUDA graph replays
+// with the parameters of the capture, so its flag epoch cannot grow from replay to replay:
+// this kernel, captured in front of it, clears the own flags, both sets of head counters and
+// both status slots instead, and any epoch above zero then means "published by this run".
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+entwine_reset_kernel(unsigned* flags, int n_flags, int* heads, int n_heads, StatusSlot* status) {
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  for (int i = tid; i < n_flags; i += nth) flags[i] = 0;
+  for (int i = tid; i < n_heads; i += nth) heads[i] = 0;
+  if (tid < 2) {
+    StatusSlot* s = &status[tid];
+    s->code_cta_task = 0;
+    s->flags_published = 0;
+    s->tiles_reduced = 0;
+    s->tiles_pushed = 0;
+    s->t_start = ~0ULL;
+    s->t_gemm_end = 0;
+    s->t_end = 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------
 // NORM: the layer-chain variant (residual add + RMSNorm in the consumer) is a kernel of its own,
@@ -1587,6 +1610,7 @@ struct DeviceState {
   unsigned* band_ctr = nullptr;  // layer chain: [rowsT]
   unsigned epoch = 0;
   unsigned seq = 0;
+  bool captured = false;  // a launch of this plan has been captured into a CUDA graph
   bool status_pending = false;
   cudaStream_t last_stream = nullptr;
   int64_t withheld = -1;
@@ -1847,6 +1871,12 @@ struct NormArgs {
 
 static int launch(Plan* p, int mode, const void* A, const void* B, const void* partial, const void* peers,
                   void* out, void* send, int n_ctas, cudaStream_t stream, const NormArgs* norm = nullptr) {
+  if (!p->dev || !p->launched) {
+    // the first launch allocates the workspace and configures the kernel: not inside a capture
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone)
+      return ENTWINE_ERR_INVALID;
+  }
   int rc = ensure_device(p);
   if (rc != ENTWINE_OK) return rc;
   DeviceState* d = p->dev;
@@ -1859,6 +1889,9 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
     // a CTA that waits for a band cannot drain lists: every list needs a consumer CTA of its own
     if (p->x > p->n_gemm_ctas + p->n_comm_ctas) return ENTWINE_ERR_INVALID;
     if (!d->ssq_part) {
+      cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+      if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone)
+        return ENTWINE_ERR_INVALID;  // the layer chain's scratch is allocated by an eager call
       if (cudaMalloc(&d->ssq_part, size_t(g.R) * g.nTn * 4) != cudaSuccess ||
           cudaMalloc(&d->band_ctr, size_t(g.rowsT) * 4) != cudaSuccess) {
         cudaGetLastError();
@@ -1872,8 +1905,20 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
     return ENTWINE_ERR_INVALID;
   if (partial && !aligned16(partial)) return ENTWINE_ERR_INVALID;
 
-  // serialise with the plan's previous launch if the caller switched streams
-  if (d->last_stream != stream && p->launched) CK(cudaStreamSynchronize(d->last_stream));
+  // A launch may be captured into a CUDA graph once the plan has run eagerly (nothing is
+  // allocated or configured during a capture).  From then on every launch of the plan, replayed
+  // or not, starts with the reset kernel.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  CK(cudaStreamIsCapturing(stream, &cap));
+  const bool capturing = cap != cudaStreamCaptureStatusNone;
+  if (capturing) {
+    if (!p->launched || (norm && !d->ssq_part)) return ENTWINE_ERR_INVALID;
+    d->captured = true;
+  }
+
+  // serialise with the plan's previous launch if the caller switched streams (a graph's
+  // launches are ordered by whoever replays it)
+  if (d->last_stream != stream && p->launched && !capturing) CK(cudaStreamSynchronize(d->last_stream));
 
   if (mode != MODE_COMM_ONLY) {
     d->epoch += 1;
@@ -1898,6 +1943,12 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
       CK(cudaMemsetAsync(d->flags_peer + q * g.Q + t, 0, 4, stream));
     }
     d->withheld = p->withhold_peer;
+  }
+  if (d->captured) {
+    const int n_flags = g.W * int(g.Q), n_heads = 2 * (p->x + 1);
+    const int blocks = std::min(64, (std::max(n_flags, n_heads) + 1023) / 1024);
+    entwine_reset_kernel<<<blocks, 1024, 0, stream>>>(d->flags_own, n_flags, d->list_head, n_heads, d->status);
+    CK(cudaGetLastError());
   }
 
   KParams kp;
@@ -1999,7 +2050,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   if (rc != ENTWINE_OK) return rc;
   d->seq = seq_next;
   p->launched = true;
-  d->last_stream = stream;
+  if (!capturing) d->last_stream = stream;
   d->status_pending = true;
   return ENTWINE_OK;
 }
