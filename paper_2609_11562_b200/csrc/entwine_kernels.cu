@@ -1874,8 +1874,11 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   if (!p->dev || !p->launched) {
     // the first launch allocates the workspace and configures the kernel: not inside a capture
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone)
-      return ENTWINE_ERR_INVALID;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) {
+      cudaGetLastError();
+      return ENTWINE_ERR_CUDA;
+    }
+    if (cs != cudaStreamCaptureStatusNone) return ENTWINE_ERR_INVALID;
   }
   int rc = ensure_device(p);
   if (rc != ENTWINE_OK) return rc;
