@@ -290,6 +290,40 @@ int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const void* B,
                            const void* peer_partials, void* out_shard, void* send_bufs,
                            void* stream, int64_t* status_out);
 
+/*
+ * entwine_heap_bytes / entwine_gemm_rs_pull - the call of one rank when the W ranks run on GPUs
+ * of their own (Sec. 4.1: partial outputs and flags live in a symmetric heap; Sec. 4.2: the
+ * reducer waits for the flags of all W contributions and reads the peers' tiles itself).
+ *
+ * The heap is W segments, segment w belonging to rank w, mapped by every rank so that segment
+ * w starts at heap + w * heap_stride (device pointer valid on the calling rank's GPU: its own
+ * memory for w = rank, peer-mapped memory otherwise).  entwine_heap_bytes gives the least
+ * size of a segment and, optionally, where its flag array starts; heap and heap_stride must
+ * be multiples of 256 bytes, and the whole heap must be zero before the first call.
+ * A segment holds two partial-output buffers [M][N] (bf16), used alternately by the parity of
+ * `epoch`, and the flags [W sources][Q] (uint32) that the W ranks write for this rank's tiles.
+ *
+ * entwine_gemm_rs_pull(plan, A, B, heap, heap_stride, epoch, produce_only, out_shard, stream):
+ * the producer stores the rank's partial into its own segment and, per finished tile, writes
+ * `epoch` into the flag array of the tile's destination rank (a store into that rank's
+ * segment, system scope); the consumer warps reduce the tiles of the rank's own partition:
+ * they poll the rank's local flags until all W sources show a value >= epoch and read the W
+ * contributions (own segment first, then the peers' in ascending rank order) into
+ * out_shard[R][N].  There are no push tasks and no send buffers: the peers' reads are the
+ * communication of Eq. 2.  `epoch` is the call's sequence number: the same on every rank,
+ * 1, 2, 3, ... without gaps.  Two buffers suffice because a rank can finish call n+1 only
+ * after every peer has started it, i.e. finished reading the buffers of call n.
+ * produce_only != 0 runs the producer alone (out_shard may be NULL).
+ * Not available: coarse release groups, the layer chain, capture into a CUDA graph (the
+ * epoch is a launch parameter).  Errors as entwine_gemm_rs.
+ * On one GPU the call is exercised rank by rank: a rank's consumer never waits for a kernel
+ * that has not been launched if the other ranks' producers have run before it.
+ */
+int entwine_heap_bytes(entwine_plan_t plan, int64_t* segment_bytes, int64_t* flags_offset);
+int entwine_gemm_rs_pull(entwine_plan_t plan, const void* A, const void* B, void* heap,
+                         int64_t heap_stride, uint32_t epoch, int produce_only, void* out_shard,
+                         void* stream);
+
 /* entwine_destroy - free the plan and everything it owns (synchronises its last stream). */
 int entwine_destroy(entwine_plan_t plan);
 

@@ -39,6 +39,8 @@ struct HostTables {
   std::vector<int64_t> tasks;      // [n_tasks][8]
   std::vector<int64_t> peer_offs;  // [n_reduce][W-1]
   std::vector<Task> dev_tasks;     // [n_tasks], same rows as `tasks`
+  std::vector<Task> pull_tasks;          // pull mode: the reduce tasks of dev_tasks, list by list
+  std::vector<int32_t> pull_list_offs;   // [x+1]
   int64_t counts[16] = {0};
 };
 

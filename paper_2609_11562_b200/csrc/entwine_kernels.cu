@@ -121,6 +121,12 @@ struct KParams {
   __nv_bfloat16* norm_out;        // [R][N]
   float* ssq_part;                // [R][nTn] sum of squares of a row's 128 elements inside one tile
   unsigned* band_ctr;             // [rowsT] reduced tiles per band of 128 rows (cleared per launch)
+  // pull mode (ranks on GPUs of their own, Sec. 4.2): every rank's segment of the symmetric heap
+  // lies heap_stride bytes after the previous rank's; flags_own and flags_peer both point at
+  // this rank's flag array [W sources][Q] inside its segment
+  char* heap;                    // rank 0's segment
+  long long heap_stride;
+  long long heap_flags_off;      // offset of the flag array inside a segment
   int* list_head;                // [x + 1] head counters of this launch; entry x: normalisation tasks
   int* list_head_next;           // [x] head counters of the next launch, rewound by this one (or null)
   StatusSlot* status_next;       // status slot of the next launch, cleared by this one (or null)
@@ -140,6 +146,7 @@ struct KMaps {
   CUtensorMap c_push[2];    // partial C, box 128 x prs: one load per push step
   CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N], box 128 x prs: one store per push step
   CUtensorMap p_pf;         // incoming partials, whole-tile box, for L2 prefetch
+  CUtensorMap p_hi[2];      // pull mode: partials of the ranks above this one (p_ld: the ranks below)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -373,6 +380,35 @@ __device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_re
 __device__ __forceinline__ void st_relaxed_gpu(unsigned* p, unsigned v) {
   asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+// system scope: flags that another GPU writes or reads (pull mode)
+__device__ __forceinline__ unsigned ld_relaxed_sys(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_acq_rel_sys() { asm volatile("fence.acq_rel.sys;" ::: "memory"); }
+__device__ __forceinline__ void st_relaxed_sys(unsigned* p, unsigned v) {
+  asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+template <bool SYS>
+__device__ __forceinline__ unsigned ld_relaxed_flag(const unsigned* p) {
+  return SYS ? ld_relaxed_sys(p) : ld_relaxed_gpu(p);
+}
+template <bool SYS>
+__device__ __forceinline__ unsigned ld_acquire_flag(const unsigned* p) {
+  return SYS ? ld_acquire_sys(p) : ld_acquire_gpu(p);
+}
+template <bool SYS>
+__device__ __forceinline__ void fence_acq_rel_flag() {
+  if (SYS) fence_acq_rel_sys();
+  else fence_acq_rel_gpu();
+}
+
 __device__ __forceinline__ void st_release_gpu(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -483,11 +519,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const K
 }
 
 // Bounded acquire-poll of one flag (Sec. 4.2: acquire loads until the flag is published).
+template <bool SYS = false>
 __device__ __forceinline__ bool wait_flag(const unsigned* f, const KParams& P) {
-  if (ld_acquire_gpu(f) >= P.epoch) return true;
+  if (ld_acquire_flag<SYS>(f) >= P.epoch) return true;
   unsigned long long t0 = 0;
   for (uint32_t spins = 1;; ++spins) {
-    if (ld_acquire_gpu(f) >= P.epoch) return true;
+    if (ld_acquire_flag<SYS>(f) >= P.epoch) return true;
     if ((spins % 32) == 0) {
       if (global_abort(P)) return false;
       unsigned long long now = globaltimer_ns();
@@ -731,7 +768,7 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
 // and write the result; warp 3 forwards pushed tiles with TMA stores and recycles the slots.
 // In a producer CTA the pipeline starts on the small ring A beside the producer's buffers and
 // moves to ring B (the producer's buffers) once `gemm_done` is set.
-template <bool NORM>
+template <bool NORM, bool PULL>
 __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
                                   int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -829,6 +866,9 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         k_t = rec.t;
       };
       load_window(0);
+      // row of peer slot q in the peers' flag array: the slot itself, or, in pull mode, the
+      // peer's rank in this rank's array of all W sources
+      auto peer_row = [&](int q) { return PULL ? q + (q >= P.r ? 1 : 0) : q; };
       unsigned pf[2] = {0u, 0u};
       int pf_start = -1;
       // relaxed look at the flags of the claim starting at s (if its records are in the window)
@@ -846,8 +886,8 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           const int t = __shfl_sync(0xffffffffu, k_t, src);
           pf[r] = 0xffffffffu;
           if (c < n_claim && s + c < len && kind >= 0) {
-            if (q == 0) pf[r] = ld_relaxed_gpu(&P.flags_own[own]);
-            else if (kind == 0) pf[r] = ld_relaxed_gpu(&P.flags_peer[(q - 1) * P.Q + t]);
+            if (q == 0) pf[r] = ld_relaxed_flag<PULL>(&P.flags_own[own]);
+            else if (kind == 0) pf[r] = ld_relaxed_flag<PULL>(&P.flags_peer[peer_row(q - 1) * P.Q + t]);
           }
         }
       };
@@ -866,7 +906,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           }
           ready = ~__reduce_or_sync(0xffffffffu, unset) & ((1u << n) - 1u);
           if (ready) {
-            fence_acq_rel_gpu();  // relaxed reads of published flags + this fence = acquire
+            fence_acq_rel_flag<PULL>();  // relaxed reads of published flags + this fence = acquire
             fence_async_all();    // and the TMA reads below are ordered after it
           }
         }
@@ -891,7 +931,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             if (lane == 0) report(P, -ENTWINE_ERR_INTERNAL, base + i);
             continue;
           }
-          if (P.prefetch && i + 1 < len && src + 1 < 32) {
+          if (!PULL && P.prefetch && i + 1 < len && src + 1 < 32) {
             // Look-ahead: if the list's next task is a reduce task whose peer contributions are
             // already published, pull their tiles into L2 now (one lane per peer) so that the
             // ring's loads find them there while holding a slot.  (The task may end up with
@@ -913,10 +953,10 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             const int own = __shfl_sync(0xffffffffu, k_own, src);
             const int t = __shfl_sync(0xffffffffu, k_t, src);
             bool mine_ok = true;
-            if (lane == 0) mine_ok = wait_flag(&P.flags_own[own], P);
+            if (lane == 0) mine_ok = wait_flag<PULL>(&P.flags_own[own], P);
             else if (kind == 0) {
               for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
-                mine_ok = wait_flag(&P.flags_peer[q * P.Q + t], P);
+                mine_ok = wait_flag<PULL>(&P.flags_peer[peer_row(q) * P.Q + t], P);
             }
             ok = __all_sync(0xffffffffu, mine_ok);
             if (!ok) {
@@ -966,8 +1006,19 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
                 // rs rows of the local contribution, then of all peers in ascending rank order
                 // as one 3-D box
                 tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
-                tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
-                                 ring.full(slot), pol);
+                if (!PULL) {
+                  tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
+                                   ring.full(slot), pol);
+                } else {
+                  // the peers' rows come straight from their segments of the heap: the ranks
+                  // below this one, then the ranks above it, each group as one 3-D box
+                  if (P.r > 0)
+                    tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
+                                     ring.full(slot), pol);
+                  if (P.r < P.W - 1)
+                    tma_load_3d_hint(dst + (1 + P.r) * ring.sub_bytes, &maps.p_hi[ring.geom], col,
+                                     src_row + step * rows, 0, ring.full(slot), pol);
+                }
 
               } else {
                 tma_load_2d_hint(dst, &maps.c_push[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
@@ -1167,7 +1218,7 @@ entwine_reset_kernel(unsigned* flags, int n_flags, int* heads, int n_heads, Stat
 // ------------------------------------------------------------------------------------------
 // NORM: the layer-chain variant (residual add + RMSNorm in the consumer) is a kernel of its own,
 // so that the plain kernel's code and register allocation are untouched by it.
-template <int BN, bool PAIR, bool NORM>
+template <int BN, bool PAIR, bool NORM, bool PULL>
 __global__ void __launch_bounds__(kThreads, 1)
 entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   using C = Cfg<BN, PAIR>;
@@ -1456,7 +1507,13 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       unsigned long long t0 = 0;
       auto release_block = [&](int dd, int ll) {
         const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb;
-        for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
+        if (PULL && dd != P.r) {
+          // the flag goes to its reader: row r of destination dd's flag array
+          unsigned* f = reinterpret_cast<unsigned*>(P.heap + dd * P.heap_stride + P.heap_flags_off) + P.r * P.Q;
+          for (int c = 0; c < P.cpb; ++c) st_relaxed_sys(&f[t_first + c], P.epoch);
+        } else {
+          for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
+        }
         published += P.cpb;
       };
       for (int i = 0; i < n_my; ++i) {
@@ -1484,7 +1541,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           if (seen > i) {
             t0 = 0;
             fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
-            fence_acq_rel_gpu();  // the stores seen complete by the store thread, then the flags
+            fence_acq_rel_flag<PULL>();  // the stores seen complete by the store thread, then the flags
             if (P.release_group == 1) {
               release_block(d, l);
               verdict = 1;
@@ -1580,7 +1637,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       }
     }
     if (count > 0 && !sh.abort) {
-      consumer_pipeline<NORM>(P, maps, &sh, smem_base, first, count, on_a, &cnt);
+      consumer_pipeline<NORM, PULL>(P, maps, &sh, smem_base, first, count, on_a, &cnt);
     }
     if (warp == kCommWarp && lane == 0) {
       if (cnt.reduced) atomicAdd(&st->tiles_reduced, (unsigned long long)cnt.reduced);
@@ -1606,6 +1663,8 @@ struct DeviceState {
   int* list_head = nullptr;
   StatusSlot* status = nullptr;
   unsigned* group_ctr = nullptr;
+  Task* tasks_pull = nullptr;     // pull mode: the reduce tasks alone, and their lists
+  int* list_offs_pull = nullptr;
   float* ssq_part = nullptr;     // layer chain: [R][nTn]
   unsigned* band_ctr = nullptr;  // layer chain: [rowsT]
   unsigned epoch = 0;
@@ -1656,11 +1715,12 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
 
 // 3-D map over bf16 [planes][rows][cols] with a (box_planes x box_rows x box_cols) box, no swizzle.
 static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_t rows, int64_t cols,
-                      int box_cols, int box_rows, int box_planes) {
+                      int box_cols, int box_rows, int box_planes, int64_t plane_stride_bytes = 0) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {cuuint64_t(cols), cuuint64_t(rows), cuuint64_t(planes)};
   cuuint64_t strides[2] = {cuuint64_t(cols) * 2, cuuint64_t(cols) * cuuint64_t(rows) * 2};
+  if (plane_stride_bytes > 0) strides[1] = cuuint64_t(plane_stride_bytes);
   cuuint32_t box[3] = {cuuint32_t(box_cols), cuuint32_t(box_rows), cuuint32_t(box_planes)};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
@@ -1760,6 +1820,8 @@ void device_release(Plan* p) {
   cudaFree(d->list_head);
   cudaFree(d->status);
   cudaFree(d->group_ctr);
+  cudaFree(d->tasks_pull);
+  cudaFree(d->list_offs_pull);
   cudaFree(d->ssq_part);
   cudaFree(d->band_ctr);
   cudaFree(d->sA);
@@ -1774,16 +1836,16 @@ void device_release(Plan* p) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-template <int BN, bool PAIR, bool NORM = false>
+template <int BN, bool PAIR, bool NORM = false, bool PULL = false>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
-  if (!NORM && kp.norm) return launch_bn<BN, PAIR, true>(p, kp, maps, grid, stream);
+  if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false>(p, kp, maps, grid, stream);
   // per device: the shared-memory opt-in has been set, and how many clusters fit at once
   static int max_clusters[64] = {0};
   static bool configured[64] = {false};
   int dev = 0;
   CK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ENTWINE_ERR_RESOURCES;
-  auto kern = entwine_fused_kernel<BN, PAIR, NORM>;
+  auto kern = entwine_fused_kernel<BN, PAIR, NORM, PULL>;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(unsigned(grid), 1, 1);
@@ -2058,6 +2120,152 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   return ENTWINE_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------
+// Pull mode: the call of one rank of W ranks that run on GPUs of their own (Sec. 4.2, Sec. 4.1's
+// symmetric heap).  Every rank owns one segment of a heap that all ranks map at the same
+// stride; a segment holds two partial-output buffers [M][N] (used alternately, by the parity
+// of the call number) and the rank's flag array [W sources][Q].  The producer stores its
+// partial into its own segment and writes each tile's flag into the flag array of the tile's
+// destination; the reducers poll their local flags and read the peers' rows of their own
+// partition straight out of the peers' segments.  Nothing is pushed.
+// ------------------------------------------------------------------------------------------
+static int64_t heap_flags_offset(const Geometry& g) { return 2 * g.M * g.N * 2; }
+static int64_t heap_segment_bytes(const Geometry& g) {
+  return heap_flags_offset(g) + ((int64_t(g.W) * g.Q * 4 + 255) / 256) * 256;
+}
+
+static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_t stride, uint32_t epoch,
+                       int produce_only, void* out, cudaStream_t stream) {
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) {
+    cudaGetLastError();
+    return ENTWINE_ERR_CUDA;
+  }
+  if (cap != cudaStreamCaptureStatusNone) return ENTWINE_ERR_INVALID;  // the epoch is a launch parameter
+  int rc = ensure_device(p);
+  if (rc != ENTWINE_OK) return rc;
+  DeviceState* d = p->dev;
+  const Geometry& g = p->g;
+  const HostTables& t = p->tables;
+  if (!A || !B || !heap || !aligned16(A) || !aligned16(B) || (!produce_only && (!out || !aligned16(out))))
+    return ENTWINE_ERR_INVALID;
+  if ((reinterpret_cast<uintptr_t>(heap) & 255) || (stride & 255) || stride < heap_segment_bytes(g) ||
+      epoch == 0 || epoch >= 0xfffffff0u)
+    return ENTWINE_ERR_INVALID;
+  if (p->release_group != 1 || p->poison || p->withhold_peer >= 0) return ENTWINE_ERR_INVALID;
+  if (!d->tasks_pull) {
+    bool ok = cudaMalloc(&d->tasks_pull, std::max<size_t>(1, t.pull_tasks.size()) * sizeof(Task)) == cudaSuccess &&
+              cudaMalloc(&d->list_offs_pull, t.pull_list_offs.size() * 4) == cudaSuccess &&
+              cudaMemcpy(d->tasks_pull, t.pull_tasks.data(), t.pull_tasks.size() * sizeof(Task),
+                         cudaMemcpyHostToDevice) == cudaSuccess &&
+              cudaMemcpy(d->list_offs_pull, t.pull_list_offs.data(), t.pull_list_offs.size() * 4,
+                         cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      cudaFree(d->tasks_pull);
+      cudaFree(d->list_offs_pull);
+      d->tasks_pull = nullptr;
+      d->list_offs_pull = nullptr;
+      return ENTWINE_ERR_CUDA;
+    }
+  }
+  if (d->last_stream != stream && p->launched) CK(cudaStreamSynchronize(d->last_stream));
+  if (d->captured) {
+    // (the plan's own flags are not used here; heads and status are)
+    const int n_heads = 2 * (p->x + 1);
+    entwine_reset_kernel<<<1, 1024, 0, stream>>>(d->flags_own, 0, d->list_head, n_heads, d->status);
+    CK(cudaGetLastError());
+  }
+
+  char* seg0 = static_cast<char*>(heap);
+  char* own_seg = seg0 + int64_t(p->rank) * stride;
+  const int64_t buf_off = int64_t(epoch & 1u) * g.M * g.N * 2;
+
+  KParams kp;
+  std::memset(&kp, 0, sizeof(kp));
+  kp.M = int(g.M); kp.N = int(g.N); kp.K = int(g.K); kp.W = g.W; kp.r = p->rank; kp.order = p->order;
+  kp.rowsT = g.rowsT; kp.nBn = g.nBn; kp.nTn = g.nTn; kp.Lb = g.Lb; kp.P_blk = g.P_blk; kp.Q = g.Q;
+  kp.cpb = g.cpb; kp.R = g.R;
+  kp.x = p->x;
+  kp.mode = produce_only ? MODE_GEMM_ONLY : MODE_FUSED;
+  kp.help = (p->tail_help || p->lists_opt > 0) ? 1 : 0;
+  kp.release_group = 1;
+  kp.claim = claim_size(g.W);
+  kp.epoch = epoch;
+  const unsigned seq_next = d->seq + 1;
+  kp.seq = seq_next;
+  kp.list_head = d->list_head + size_t(seq_next & 1) * (p->x + 1);
+  kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
+  kp.status_next = &d->status[(seq_next & 1) ^ 1];
+  kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
+  rc = ring_geometry(p, &kp);
+  if (rc != ENTWINE_OK) return rc;
+  kp.colocate = p->colocate;
+  kp.prefetch = 0;
+  kp.l2_hints = p->l2_hints;
+  kp.out = static_cast<__nv_bfloat16*>(out);
+  kp.heap = seg0;
+  kp.heap_stride = stride;
+  kp.heap_flags_off = heap_flags_offset(g);
+  kp.flags_own = reinterpret_cast<unsigned*>(own_seg + kp.heap_flags_off);
+  kp.flags_peer = kp.flags_own;
+  kp.tasks = d->tasks_pull;
+  kp.list_offs = d->list_offs_pull;
+  kp.status = d->status;
+
+  int grid;
+  const bool pair = p->pair;
+  if (!produce_only) {
+    kp.n_ded = p->n_comm_ctas;
+    kp.G = p->n_gemm_ctas;
+    grid = p->n_comm_ctas + p->n_gemm_ctas;
+  } else {
+    kp.n_ded = 0;
+    kp.G = pair ? (p->num_sms & ~1) : p->num_sms;
+    grid = kp.G;
+  }
+  if (pair && (grid & 1)) {
+    if (grid + 1 > p->num_sms) grid -= 1, kp.n_ded -= 1;
+    else grid += 1, kp.n_ded += 1;
+    if (kp.n_ded < p->x) kp.help = 1;
+  }
+
+  KMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  void* own_buf = own_seg + buf_off;
+  const int r = p->rank, W = g.W;
+  bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
+            make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
+            make_map(&maps.c_st, own_buf, g.M, g.N, 64, kBM, true) &&
+            make_map(&maps.p_pf, own_buf, g.M, g.N, kTile, kTile, false);
+  for (int id = 0; ok && id < 2; ++id) {
+    const int rs = kp.rs[id];
+    const int prs = kp.prs[id];
+    // the ranks below this one start at rank 0's segment, the ranks above it at rank r+1's; an
+    // empty group gets a map of this rank's buffer, which no load uses
+    const void* lo = r > 0 ? seg0 + buf_off : own_buf;
+    const void* hi = r < W - 1 ? seg0 + int64_t(r + 1) * stride + buf_off : own_buf;
+    ok = make_map(&maps.c_ld[id], own_buf, g.M, g.N, kTile, rs, false) &&
+         make_map(&maps.c_push[id], own_buf, g.M, g.N, kTile, prs, false) &&
+         make_map3(&maps.p_ld[id], lo, std::max(r, 1), g.M, g.N, kTile, rs, std::max(r, 1), stride) &&
+         make_map3(&maps.p_hi[id], hi, std::max(W - 1 - r, 1), g.M, g.N, kTile, rs, std::max(W - 1 - r, 1),
+                   stride) &&
+         make_map(&maps.send_st[id], own_buf, g.M, g.N, kTile, prs, false) &&
+         make_map(&maps.res_ld[id], own_buf, g.M, g.N, kTile, prs, false);
+  }
+  if (!ok) return ENTWINE_ERR_CUDA;
+  if (pair) rc = launch_bn<256, true, false, true>(p, kp, maps, grid, stream);
+  else if (g.BN == 256) rc = launch_bn<256, false, false, true>(p, kp, maps, grid, stream);
+  else rc = launch_bn<128, false, false, true>(p, kp, maps, grid, stream);
+  if (rc != ENTWINE_OK) return rc;
+  d->seq = seq_next;
+  p->launched = true;
+  d->last_stream = stream;
+  d->status_pending = true;
+  return ENTWINE_OK;
+}
+
 }  // namespace entwine
 
 using namespace entwine;
@@ -2088,6 +2296,20 @@ int entwine_gemm_only(entwine_plan_t plan, const void* A, const void* B, void* s
   if (!plan) return ENTWINE_ERR_INVALID;
   return launch(plan, MODE_GEMM_ONLY, A, B, nullptr, nullptr, nullptr, nullptr, 0,
                 static_cast<cudaStream_t>(stream));
+}
+
+int entwine_heap_bytes(entwine_plan_t plan, int64_t* segment_bytes, int64_t* flags_offset) {
+  if (!plan || !segment_bytes) return ENTWINE_ERR_INVALID;
+  *segment_bytes = heap_segment_bytes(plan->g);
+  if (flags_offset) *flags_offset = heap_flags_offset(plan->g);
+  return ENTWINE_OK;
+}
+
+int entwine_gemm_rs_pull(entwine_plan_t plan, const void* A, const void* B, void* heap, int64_t heap_stride,
+                         uint32_t epoch, int produce_only, void* out_shard, void* stream) {
+  if (!plan) return ENTWINE_ERR_INVALID;
+  return launch_pull(plan, A, B, heap, heap_stride, epoch, produce_only, out_shard,
+                     static_cast<cudaStream_t>(stream));
 }
 
 int entwine_comm_only(entwine_plan_t plan, const void* partial, const void* peer_partials, void* out_shard,

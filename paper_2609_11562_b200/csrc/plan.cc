@@ -95,6 +95,8 @@ void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, i
     }
   }
 
+  out->pull_list_offs.assign(size_t(x) + 1, 0);
+  out->pull_tasks.clear();
   out->list_offs.assign(size_t(x) + 1, 0);
   out->tasks.clear();
   out->peer_offs.clear();
@@ -115,6 +117,7 @@ void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, i
       dt.kind = e.kind; dt.d = e.d; dt.t = e.t; dt.slot = slot;
       dt.src_off = src; dt.dst_off = dst;
       out->dev_tasks.push_back(dt);
+      if (e.kind == 0) out->pull_tasks.push_back(dt);
       if (e.kind == 0) {
         for (int w = 0; w < W; ++w) {
           if (w == r) continue;
@@ -127,6 +130,7 @@ void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, i
       }
     }
     out->list_offs[size_t(j) + 1] = int32_t(out->dev_tasks.size());
+    out->pull_list_offs[size_t(j) + 1] = int32_t(out->pull_tasks.size());
   }
 
   const int64_t tile_bytes = int64_t(kTile) * kTile * 2;

@@ -34,13 +34,15 @@ RELEASE_PARTITION, RELEASE_WHOLE = -1, -2
 SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gemm_rs_host",
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
            "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static",
-           "entwine_gemm_rs_norm")
+           "entwine_gemm_rs_norm", "entwine_heap_bytes", "entwine_gemm_rs_pull")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
 _lib.entwine_set_option.argtypes = [_vp, _int, _i64]
 _lib.entwine_gemm_rs_norm.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
 _lib.entwine_gemm_rs.argtypes = [_vp] * 7
+_lib.entwine_heap_bytes.argtypes = [_vp, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]
+_lib.entwine_gemm_rs_pull.argtypes = [_vp, _vp, _vp, _vp, _i64, ctypes.c_uint32, _int, _vp, _vp]
 _lib.entwine_gemm_rs_host.argtypes = [_vp] * 6
 _lib.entwine_gemm_only.argtypes = [_vp] * 4
 _lib.entwine_comm_only.argtypes = [_vp, _vp, _vp, _vp, _vp, _int, _vp]
@@ -124,6 +126,17 @@ class Plan:
         _check(_lib.entwine_gemm_rs_norm(self._h, _ptr(A), _ptr(B), _ptr(peer_partials), _ptr(residual),
                                          _ptr(weight), float(eps), _ptr(hidden_out), _ptr(norm_out),
                                          _ptr(send_bufs), _stream(stream)), "entwine_gemm_rs_norm")
+
+    def heap_bytes(self):
+        """(least bytes of one rank's heap segment, offset of its flag array)."""
+        seg, off = _i64(0), _i64(0)
+        _check(_lib.entwine_heap_bytes(self._h, ctypes.byref(seg), ctypes.byref(off)), "entwine_heap_bytes")
+        return seg.value, off.value
+
+    def gemm_rs_pull(self, A, B, heap, heap_stride, epoch, out_shard, produce_only=False, stream=None):
+        _check(_lib.entwine_gemm_rs_pull(self._h, _ptr(A), _ptr(B), _ptr(heap), int(heap_stride), int(epoch),
+                                         1 if produce_only else 0, _ptr(out_shard), _stream(stream)),
+               "entwine_gemm_rs_pull")
 
     def gemm_rs_host(self, A, B, peer_partials, out_shard, send_bufs):
         """Host tensors (CPU, bf16, contiguous; pinned for speed)."""
