@@ -314,6 +314,32 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
                                            flush, torch)
         plan0.destroy()
         del Cfull
+        # Pull mode (the rank's call when the W ranks have GPUs of their own): this rank's kernel
+        # with the peers' contributions already in their heap segments and flagged, this GPU's
+        # HBM standing in for the reads over NVLink.  No push tasks: a peer's pull is its own work.
+        time.sleep(0.5)
+        seg, flags_off = plan.heap_bytes()
+        heap = torch.zeros(wl.W * seg, dtype=torch.uint8, device="cuda")
+        r = launch["rank"]
+        Q = plan.counts()["Q"]
+        for w in range(wl.W):
+            if w != r:
+                heap[w * seg:w * seg + flags_off].view(torch.bfloat16).normal_()
+        fl = heap[r * seg + flags_off:r * seg + flags_off + wl.W * Q * 4].view(torch.int32).view(wl.W, Q)
+        fl.fill_(0x7fffffff)  # every peer is ahead of any call number used here
+        fl[r].zero_()         # the rank's own flags are published by each call
+        pplan = E.Plan(wl.M, wl.N, wl.K, wl.W, launch["order"], launch["n_comm_sms"], rank=r,
+                       **launch.get("opts", {}))
+        calls = [0]
+
+        def pull():
+            calls[0] += 1
+            pplan.gemm_rs_pull(A, Bm, heap, seg, calls[0], out)
+        res["pull_us"] = time_steps(pull, max(5, steps // 4), 3, flush, torch)
+        st = pplan.last_status()
+        assert st["tiles_reduced"] == pplan.counts()["n_reduce"] and st["tiles_pushed"] == 0
+        pplan.destroy()
+        del heap, fl
     plan.destroy()
     return res
 
@@ -728,6 +754,7 @@ def main():
                 "gemm_alone_us": med(r["gemm_only_us"]),
                 "comm_alone_all_sms_us": med(r["comm_only_us"]),
                 "comm_alone_GBps": w2.comm_bytes / med(r["comm_only_us"]) / 1e3,
+                "pull_mode_us": med(r["pull_us"]),
                 "overlap_efficiency": med(r["gemm_only_us"]) / fused,
                 "tail_us": (r["status"]["t_end_ns"] - r["status"]["t_gemm_ns"]) / 1e3,
                 "n_comm_sms": LAUNCH[name]["n_comm_sms"],
