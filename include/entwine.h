@@ -191,6 +191,21 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B,
                          const void* peer_partials, void* out_shard, void* send_bufs);
 
 /*
+ * entwine_gemm_rs_host_begin / entwine_gemm_rs_host_wait - the host-buffer call as a pipeline
+ * of depth two.  _begin enqueues the copies up, the fused call and the copies down of one call
+ * on streams of the library (two staging sets on the device, used alternately) and returns;
+ * _wait blocks until the oldest call that has not been waited for has delivered out_shard and
+ * send_bufs (and returns at once if there is none).  With pinned host buffers the copies up
+ * of one call overlap the copies down of the call before it.  At most two calls may be
+ * outstanding: a third _begin without a _wait returns ENTWINE_ERR_INVALID.  The host buffers
+ * of a call must stay untouched until its _wait.  Device-side failures are reported by
+ * entwine_last_status, as for entwine_gemm_rs.
+ */
+int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B,
+                               const void* peer_partials, void* out_shard, void* send_bufs);
+int entwine_gemm_rs_host_wait(entwine_plan_t plan);
+
+/*
  * entwine_gemm_rs_norm - the fused call followed, inside the same launch, by the rest of the
  * attention-output layer's chain (Sec. 5.2.3: GEMM + ReduceScatter, then residual addition and
  * RMSNorm).  The reduction of an owned tile adds residual[R][N] to the rank-order fp32 sum and

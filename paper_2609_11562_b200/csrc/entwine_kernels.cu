@@ -1675,6 +1675,15 @@ struct DeviceState {
   int64_t withheld = -1;
   // staging for the host-buffer entry point
   cudaStream_t own_stream = nullptr;
+  // pipelined host-buffer calls: two staging sets, copies up and down on streams of their own
+  struct HostPipe {
+    cudaStream_t up = nullptr, comp = nullptr, down = nullptr;
+    cudaEvent_t up_done[2] = {nullptr, nullptr}, k_done[2] = {nullptr, nullptr}, d_done[2] = {nullptr, nullptr};
+    __nv_bfloat16 *A[2] = {nullptr, nullptr}, *B[2] = {nullptr, nullptr}, *peers[2] = {nullptr, nullptr};
+    __nv_bfloat16 *out[2] = {nullptr, nullptr}, *send[2] = {nullptr, nullptr};
+    uint64_t issued = 0, waited = 0;
+  };
+  HostPipe* pipe = nullptr;
   __nv_bfloat16 *sA = nullptr, *sB = nullptr, *sPeers = nullptr, *sOut = nullptr, *sSend = nullptr;
 };
 
@@ -1808,6 +1817,27 @@ void device_release(Plan* p) {
   DeviceState* d = p->dev;
   if (!d) return;
   if (d->last_stream || d->status_pending) cudaStreamSynchronize(d->last_stream);
+  if (d->pipe) {
+    DeviceState::HostPipe* hp = d->pipe;
+    for (cudaStream_t st : {hp->up, hp->comp, hp->down}) {
+      if (st) {
+        cudaStreamSynchronize(st);
+        cudaStreamDestroy(st);
+      }
+    }
+    for (int i = 0; i < 2; ++i) {
+      if (hp->up_done[i]) cudaEventDestroy(hp->up_done[i]);
+      if (hp->k_done[i]) cudaEventDestroy(hp->k_done[i]);
+      if (hp->d_done[i]) cudaEventDestroy(hp->d_done[i]);
+      cudaFree(hp->A[i]);
+      cudaFree(hp->B[i]);
+      cudaFree(hp->peers[i]);
+      cudaFree(hp->out[i]);
+      cudaFree(hp->send[i]);
+    }
+    delete hp;
+    d->pipe = nullptr;
+  }
   if (d->own_stream) {
     cudaStreamSynchronize(d->own_stream);
     cudaStreamDestroy(d->own_stream);
@@ -2395,6 +2425,74 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, cons
   CK(cudaStreamSynchronize(s));
   int64_t stw[8];
   return entwine_last_status(plan, stw);
+}
+
+int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B, const void* peer_partials,
+                               void* out_shard, void* send_bufs) {
+  if (!plan || !A || !B || !peer_partials || !out_shard || !send_bufs) return ENTWINE_ERR_INVALID;
+  int rc = ensure_device(plan);
+  if (rc != ENTWINE_OK) return rc;
+  DeviceState* d = plan->dev;
+  const Geometry& g = plan->g;
+  const size_t szA = size_t(g.M) * g.K * 2, szB = size_t(g.N) * g.K * 2;
+  const size_t szP = size_t(g.W - 1) * g.M * g.N * 2, szO = size_t(g.R) * g.N * 2;
+  const size_t szS = size_t(g.W - 1) * g.R * g.N * 2;
+  if (!d->pipe) {
+    DeviceState::HostPipe* hp = new DeviceState::HostPipe();
+    d->pipe = hp;  // released with the plan, whatever was allocated
+    bool ok = cudaStreamCreateWithFlags(&hp->up, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp->comp, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp->down, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 2; ++i) {
+      ok = cudaEventCreateWithFlags(&hp->up_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp->k_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp->d_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaMalloc(&hp->A[i], szA) == cudaSuccess && cudaMalloc(&hp->B[i], szB) == cudaSuccess &&
+           cudaMalloc(&hp->peers[i], szP) == cudaSuccess && cudaMalloc(&hp->out[i], szO) == cudaSuccess &&
+           cudaMalloc(&hp->send[i], szS) == cudaSuccess;
+    }
+    if (!ok) {
+      cudaGetLastError();
+      return ENTWINE_ERR_CUDA;
+    }
+  }
+  DeviceState::HostPipe* hp = d->pipe;
+  if (!hp->send[1]) return ENTWINE_ERR_CUDA;             // an earlier set-up failed part-way
+  if (hp->issued - hp->waited >= 2) return ENTWINE_ERR_INVALID;  // both staging sets are in use
+  const int s = int(hp->issued & 1);
+  // copies up: after the kernel that last read this staging set
+  CK(cudaStreamWaitEvent(hp->up, hp->k_done[s], 0));
+  CK(cudaMemcpyAsync(hp->A[s], A, szA, cudaMemcpyHostToDevice, hp->up));
+  CK(cudaMemcpyAsync(hp->B[s], B, szB, cudaMemcpyHostToDevice, hp->up));
+  const size_t part = size_t(g.R) * g.N * 2, full = size_t(g.M) * g.N * 2;
+  for (int q = 0; q < g.W - 1; ++q) {
+    const size_t off = size_t(q) * full + size_t(plan->rank) * part;
+    CK(cudaMemcpyAsync(reinterpret_cast<char*>(hp->peers[s]) + off, static_cast<const char*>(peer_partials) + off,
+                       part, cudaMemcpyHostToDevice, hp->up));
+  }
+  CK(cudaEventRecord(hp->up_done[s], hp->up));
+  // the kernel: after its inputs are up and the copies down that last read this set's results
+  CK(cudaStreamWaitEvent(hp->comp, hp->up_done[s], 0));
+  CK(cudaStreamWaitEvent(hp->comp, hp->d_done[s], 0));
+  rc = launch(plan, MODE_FUSED, hp->A[s], hp->B[s], nullptr, hp->peers[s], hp->out[s], hp->send[s], 0, hp->comp);
+  if (rc != ENTWINE_OK) return rc;
+  CK(cudaEventRecord(hp->k_done[s], hp->comp));
+  CK(cudaStreamWaitEvent(hp->down, hp->k_done[s], 0));
+  CK(cudaMemcpyAsync(out_shard, hp->out[s], szO, cudaMemcpyDeviceToHost, hp->down));
+  CK(cudaMemcpyAsync(send_bufs, hp->send[s], szS, cudaMemcpyDeviceToHost, hp->down));
+  CK(cudaEventRecord(hp->d_done[s], hp->down));
+  hp->issued += 1;
+  return ENTWINE_OK;
+}
+
+int entwine_gemm_rs_host_wait(entwine_plan_t plan) {
+  if (!plan) return ENTWINE_ERR_INVALID;
+  DeviceState* d = plan->dev;
+  if (!d || !d->pipe || d->pipe->waited == d->pipe->issued) return ENTWINE_OK;
+  DeviceState::HostPipe* hp = d->pipe;
+  CK(cudaEventSynchronize(hp->d_done[hp->waited & 1]));
+  hp->waited += 1;
+  return ENTWINE_OK;
 }
 
 }  // extern "C"

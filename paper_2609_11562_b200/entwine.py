@@ -34,7 +34,8 @@ RELEASE_PARTITION, RELEASE_WHOLE = -1, -2
 SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gemm_rs_host",
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
            "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static",
-           "entwine_gemm_rs_norm", "entwine_heap_bytes", "entwine_gemm_rs_pull")
+           "entwine_gemm_rs_norm", "entwine_heap_bytes", "entwine_gemm_rs_pull",
+           "entwine_gemm_rs_host_begin", "entwine_gemm_rs_host_wait")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
@@ -44,6 +45,8 @@ _lib.entwine_gemm_rs.argtypes = [_vp] * 7
 _lib.entwine_heap_bytes.argtypes = [_vp, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]
 _lib.entwine_gemm_rs_pull.argtypes = [_vp, _vp, _vp, _vp, _i64, ctypes.c_uint32, _int, _vp, _vp]
 _lib.entwine_gemm_rs_host.argtypes = [_vp] * 6
+_lib.entwine_gemm_rs_host_begin.argtypes = [_vp] * 6
+_lib.entwine_gemm_rs_host_wait.argtypes = [_vp]
 _lib.entwine_gemm_only.argtypes = [_vp] * 4
 _lib.entwine_comm_only.argtypes = [_vp, _vp, _vp, _vp, _vp, _int, _vp]
 _lib.entwine_read_partial.argtypes = [_vp, _vp, _vp]
@@ -142,6 +145,14 @@ class Plan:
         """Host tensors (CPU, bf16, contiguous; pinned for speed)."""
         _check(_lib.entwine_gemm_rs_host(self._h, _ptr(A), _ptr(B), _ptr(peer_partials),
                                          _ptr(out_shard), _ptr(send_bufs)), "entwine_gemm_rs_host")
+
+    def gemm_rs_host_begin(self, A, B, peer_partials, out_shard, send_bufs):
+        """Enqueue one host-buffer call (at most two outstanding); pair with gemm_rs_host_wait."""
+        _check(_lib.entwine_gemm_rs_host_begin(self._h, _ptr(A), _ptr(B), _ptr(peer_partials),
+                                               _ptr(out_shard), _ptr(send_bufs)), "entwine_gemm_rs_host_begin")
+
+    def gemm_rs_host_wait(self):
+        _check(_lib.entwine_gemm_rs_host_wait(self._h), "entwine_gemm_rs_host_wait")
 
     def gemm_rs_static(self, A, B, peer_partials, out_shard, send_bufs, stream=None, want_status=True):
         """The fused call on the library's fixed scratch array: for callers that must not
