@@ -32,7 +32,7 @@ METRIC = "fused GEMM-RS TFLOP/s and fraction of max(tensor peak, HBM) roofline"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic (bytes read + written per launch) of the fused kernel from an ncu capture of
 # the named workload; see profiles/.  None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"attn_out_proj": 53.69e6, "mlp_down_proj": 834.54e6, "short_k_comm_bound": 517.00e6}
+NCU_TRAFFIC_BYTES = {"attn_out_proj": 53.69e6, "mlp_down_proj": 845.38e6, "short_k_comm_bound": 507.35e6}
 # Launch configuration per workload: communication SMs, tile order.
 # Launch configuration per workload (the best point of a budget x order scan on B200): number of
 # dedicated communication SMs (0 = consumer warps co-located with the producer in every CTA),
