@@ -886,7 +886,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           const int t = __shfl_sync(0xffffffffu, k_t, src);
           pf[r] = 0xffffffffu;
           if (c < n_claim && s + c < len && kind >= 0) {
-            if (q == 0) pf[r] = ld_relaxed_flag<PULL>(&P.flags_own[own]);
+            if (q == 0) pf[r] = ld_relaxed_gpu(&P.flags_own[own]);  // written by this GPU in every mode
             else if (kind == 0) pf[r] = ld_relaxed_flag<PULL>(&P.flags_peer[peer_row(q - 1) * P.Q + t]);
           }
         }
@@ -953,7 +953,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             const int own = __shfl_sync(0xffffffffu, k_own, src);
             const int t = __shfl_sync(0xffffffffu, k_t, src);
             bool mine_ok = true;
-            if (lane == 0) mine_ok = wait_flag<PULL>(&P.flags_own[own], P);
+            if (lane == 0) mine_ok = wait_flag<false>(&P.flags_own[own], P);
             else if (kind == 0) {
               for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
                 mine_ok = wait_flag<PULL>(&P.flags_peer[peer_row(q) * P.Q + t], P);
@@ -1541,7 +1541,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           if (seen > i) {
             t0 = 0;
             fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
-            fence_acq_rel_flag<PULL>();  // the stores seen complete by the store thread, then the flags
+            // the stores seen complete by the store thread, then the flags; system scope only
+            // where the flags go to another GPU
+            if (PULL && d != P.r) fence_acq_rel_sys();
+            else fence_acq_rel_gpu();
             if (P.release_group == 1) {
               release_block(d, l);
               verdict = 1;
