@@ -105,17 +105,6 @@ enum {
                                       ENTWINE_RELEASE_PARTITION (-1): all tiles of a destination
                                       partition together; ENTWINE_RELEASE_WHOLE (-2): the whole
                                       output together.  Results are identical for every value      */
-  ENTWINE_OPT_LIST_BALANCE    = 15, /* [pre] weighting of the consumer lists when every CTA first
-                                      produces (n_comm_sms = 0, one list per CTA).  The producer's
-                                      positions rarely divide evenly among the CTAs, so some CTAs
-                                      reach their consumer work one producer unit earlier.  0
-                                      (default): the paper's round-robin lists (Sec. 3.1).  b > 0: a
-                                      CTA with u fewer producer units than the busiest gets b/10 * u
-                                      more tasks; tasks are dealt in publication order to the list
-                                      with the least load for its weight (reduce = W + 1 tiles,
-                                      push = 2).  Ignored with dedicated communication SMs or
-                                      ENTWINE_OPT_LISTS.  The paper has no counterpart (its
-                                      consumer CTAs do not produce); results are identical        */
   ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */

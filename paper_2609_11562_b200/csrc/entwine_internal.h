@@ -61,7 +61,7 @@ bool make_geometry(int64_t M, int64_t N, int64_t K, int W, int BN, Geometry* g);
 // Block p of the logical order -> block row, block column, destination, within-partition index.
 void block_of_position(const Geometry& g, int order, int p, int* mb, int* nb, int* d, int* l);
 void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, int n_comm_ctas,
-                  int pair, int balance, HostTables* out);
+                  HostTables* out);
 
 // Launch modes of the one kernel.
 enum Mode { MODE_FUSED = 0, MODE_GEMM_ONLY = 1, MODE_COMM_ONLY = 2 };
@@ -79,7 +79,6 @@ struct Plan {
   int prefetch = 0;         // look-ahead L2 prefetch of peer tiles (measured: no gain)
   int l2_hints = 3;         // bit 0: evict-first on the consumer's TMA traffic, bit 1: evict-last on operands
   int lists_opt = 0;        // number of consumer lists x, 0 = one per consumer CTA
-  int list_balance = 0;     // tenths of a task a CTA gets more per producer unit it has less (0: round-robin lists)
   int release_group = 1;    // blocks released together; -1 per destination partition, -2 whole output
   int stages = 0;           // operand-ring stages of the producer, 0 = choose
   int colocate = 1;         // consumer warps of a producer CTA work while it produces

@@ -60,7 +60,7 @@ struct Pending {
 }  // namespace
 
 void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, int n_comm_ctas,
-                  int pair, int balance, HostTables* out) {
+                  HostTables* out) {
   const int P = g.P_blk, cpb = g.cpb, W = g.W, Q = g.Q;
   out->order.assign(size_t(P) * 4, 0);
   out->tiles.assign(size_t(P) * cpb, 0);
@@ -92,51 +92,6 @@ void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, i
         lists[size_t(u % x_p)].push_back({1, d, t, k});
         ++u;
       }
-    }
-  }
-
-  if (balance > 0 && n_comm_ctas == 0 && x == n_gemm_ctas) {
-    // Lists weighted by the time their CTAs have left for them.  Every CTA first produces; CTA c
-    // gets n_my(c) producer units (pair tiles or blocks), and the positions do not divide evenly,
-    // so some CTAs reach their consumer work one unit earlier than others.  A CTA with u fewer
-    // units than the busiest gets `balance`/10 * u more tasks than those.  Tasks are dealt in
-    // publication order to the list whose load, relative to its weight, stays smallest (ties:
-    // lowest list), a reduce task weighing W + 1 tiles moved and a push task 2.
-    const int n_units = pair ? g.P_blk / 2 : g.P_blk;
-    const int stride = pair ? n_gemm_ctas / 2 : n_gemm_ctas;
-    std::vector<int64_t> n_my(static_cast<size_t>(x));
-    int64_t n_max = 0;
-    for (int c = 0; c < x; ++c) {
-      const int unit0 = pair ? c / 2 : c;
-      n_my[size_t(c)] = unit0 < n_units ? (n_units - unit0 + stride - 1) / stride : 0;
-      n_max = std::max(n_max, n_my[size_t(c)]);
-    }
-    // weights in tenths of a task: the even share plus the bonus, shifted so that they sum to
-    // the number of tasks
-    const int64_t n_tasks = int64_t(g.W) * g.Q;
-    int64_t bonus_sum = 0;
-    for (int c = 0; c < x; ++c) bonus_sum += int64_t(balance) * (n_max - n_my[size_t(c)]);
-    std::vector<int64_t> w(static_cast<size_t>(x));
-    for (int c = 0; c < x; ++c) {
-      const int64_t v = (10 * n_tasks - bonus_sum) / x + int64_t(balance) * (n_max - n_my[size_t(c)]);
-      w[size_t(c)] = std::max<int64_t>(v, 1);
-    }
-    std::vector<Pending> all;
-    for (auto& lst : lists) {
-      all.insert(all.end(), lst.begin(), lst.end());
-      lst.clear();
-    }
-    std::stable_sort(all.begin(), all.end(), [](const Pending& a, const Pending& b) { return a.k < b.k; });
-    std::vector<int64_t> load(static_cast<size_t>(x), 0);
-    for (const Pending& e : all) {
-      const int64_t cost = e.kind == 0 ? g.W + 1 : 2;
-      int best = 0;
-      for (int c = 1; c < x; ++c) {
-        // (load[c] + cost) / w[c] < (load[best] + cost) / w[best]
-        if ((load[size_t(c)] + cost) * w[size_t(best)] < (load[size_t(best)] + cost) * w[size_t(c)]) best = c;
-      }
-      load[size_t(best)] += cost;
-      lists[size_t(best)].push_back(e);
     }
   }
 
@@ -221,8 +176,7 @@ int finalize_plan(Plan* p) {
     p->x = p->n_comm_sms;
   }
   if (p->lists_opt > 0) p->x = p->lists_opt;
-  build_tables(p->g, p->order, p->rank, p->x, p->n_gemm_ctas, p->n_comm_ctas, p->pair ? 1 : 0, p->list_balance,
-               &p->tables);
+  build_tables(p->g, p->order, p->rank, p->x, p->n_gemm_ctas, p->n_comm_ctas, &p->tables);
   p->tables_built = true;
   return ENTWINE_OK;
 }
@@ -313,10 +267,6 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
     case ENTWINE_OPT_LISTS:
       if (p->launched || value < 0 || value > 4096) return ENTWINE_ERR_INVALID;
       p->lists_opt = int(value);
-      return entwine::finalize_plan(p);
-    case ENTWINE_OPT_LIST_BALANCE:
-      if (p->launched || value < 0 || value > 1000) return ENTWINE_ERR_INVALID;
-      p->list_balance = int(value);
       return entwine::finalize_plan(p);
     case ENTWINE_OPT_RELEASE_GROUP:
       if (value == 0 || value < ENTWINE_RELEASE_WHOLE || value > (int64_t(1) << 24)) return ENTWINE_ERR_INVALID;

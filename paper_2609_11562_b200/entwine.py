@@ -25,7 +25,7 @@ OK, ERR_INVALID, ERR_RESOURCES, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2,
 ERR_TOO_LARGE = -6
 OPT_RANK, OPT_BLOCK_N, OPT_WAIT_BUDGET_NS, OPT_TAIL_HELP = 1, 2, 3, 4
 OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL, OPT_PAIR_CTAS, OPT_COLOCATE = 5, 6, 7, 8, 9
-OPT_PREFETCH, OPT_STAGES, OPT_L2_HINTS, OPT_LISTS, OPT_RELEASE_GROUP, OPT_LIST_BALANCE = 10, 11, 12, 13, 14, 15
+OPT_PREFETCH, OPT_STAGES, OPT_L2_HINTS, OPT_LISTS, OPT_RELEASE_GROUP = 10, 11, 12, 13, 14
 RELEASE_PARTITION, RELEASE_WHOLE = -1, -2
 (EXPORT_COUNTS, EXPORT_ORDER, EXPORT_TILES, EXPORT_FLAG_SEQ, EXPORT_LIST_OFFS, EXPORT_TASKS,
  EXPORT_PEER_OFFS) = range(7)
@@ -110,8 +110,7 @@ class Plan:
         self.rank = 0
         keys = {"rank": OPT_RANK, "block_n": OPT_BLOCK_N, "wait_budget_ns": OPT_WAIT_BUDGET_NS,
                 "tail_help": OPT_TAIL_HELP, "num_sms": OPT_NUM_SMS, "poison_partial": OPT_POISON_PARTIAL,
-                "pair_ctas": OPT_PAIR_CTAS, "colocate": OPT_COLOCATE, "prefetch": OPT_PREFETCH, "stages": OPT_STAGES, "l2_hints": OPT_L2_HINTS, "lists": OPT_LISTS, "release_group": OPT_RELEASE_GROUP,
-                "list_balance": OPT_LIST_BALANCE}
+                "pair_ctas": OPT_PAIR_CTAS, "colocate": OPT_COLOCATE, "prefetch": OPT_PREFETCH, "stages": OPT_STAGES, "l2_hints": OPT_L2_HINTS, "lists": OPT_LISTS, "release_group": OPT_RELEASE_GROUP}
         # num_sms first: it bounds the others
         for name in sorted(options, key=lambda n: n != "num_sms"):
             self.set_option(keys[name], options[name])
