@@ -151,3 +151,44 @@ def test_bad_arguments_are_refused():
         coarse.gemm_rs_pull(A, Bm, heap.mem, heap.stride, 1, out)
     plan.destroy()
     coarse.destroy()
+
+
+def test_full_size_attention_shape_rank_by_rank():
+    """The benchmark's shape (W=4, 4096 x 4096 x 1024) in pull mode, all four ranks.  Sampled
+    rows of every stored partial against the float64 oracle; for every element, each rank's
+    shard is the order-exact fp32 sum of the stored contributions (own first, peers ascending)."""
+    W, M, N, K = 4, 4096, 4096, 1024
+    R = M // W
+    plans = [E.Plan(M, N, K, W, 1, 0, rank=q) for q in range(W)]
+    heap = Heap(plans[0], W, M, N, pad=0)
+    Q = plans[0].counts()["Q"]
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([np.array([d * R, d * R + R - 1]) for d in range(W)] + [rng.integers(0, M, 40)]))
+    for epoch in (1, 2):
+        ops = [I.make_operands(I.Workload(f"pull_full{q}", W, M, N, K, "normal", "normal_fanin", 14, 4 * epoch + q),
+                               device="cuda") for q in range(W)]
+        for q in range(W):
+            plans[q].gemm_rs_pull(ops[q][0], ops[q][1], heap.mem, heap.stride, epoch, None, produce_only=True)
+            plans[q].last_status()
+        torch.cuda.synchronize()
+        stored = [heap.partial(q, epoch).clone() for q in range(W)]
+        for q in range(W):
+            Ab, Bb = I.bits(ops[q][0][rows]), I.bits(ops[q][1])
+            C_rows, S_rows = O.partial_gemm(Ab, Bb), O.abs_gemm(Ab, Bb)
+            got = O.bf16_bits_to_f64(I.bits(stored[q][rows]))
+            assert (np.abs(got - C_rows) <= O.tolerance(C_rows, S_rows)).all()
+        for k in range(W):
+            assert bool((heap.flags(k, Q) == epoch).all())
+            heap.flags(k, Q)[k].zero_()
+            out = torch.full((R, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            plans[k].gemm_rs_pull(ops[k][0], ops[k][1], heap.mem, heap.stride, epoch, out)
+            st = plans[k].last_status()
+            assert st["tiles_reduced"] == plans[k].counts()["n_reduce"] and st["tiles_pushed"] == 0
+            assert torch.equal(heap.partial(k, epoch), stored[k])
+            acc = stored[k][k * R:(k + 1) * R].float()
+            for q in range(W):
+                if q != k:
+                    acc = acc + stored[q][k * R:(k + 1) * R].float()
+            assert torch.equal(out, acc.to(torch.bfloat16))
+    for p in plans:
+        p.destroy()
