@@ -147,6 +147,7 @@ struct KMaps {
   CUtensorMap send_st[2];   // send_bufs viewed as [(W-1)*R, N], box 128 x prs: one store per push step
   CUtensorMap p_pf;         // incoming partials, whole-tile box, for L2 prefetch
   CUtensorMap p_hi[2];      // pull mode: partials of the ranks above this one (p_ld: the ranks below)
+  CUtensorMap h_ld[2];      // layer chain: hidden_out [R, N], box 128 x prs (rows of a tile to normalise)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -701,17 +702,19 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
         if (g >= g0 && g < g1) resv[k] = ld_shared_v4(sbase + (g - g0) * 16);
       }
     } else if (NORM && m.kind == 2) {
-      // Normalisation of one 128 x 128 tile of a complete band: 1/RMS of each of its rows from
-      // the nTn partial sums (fixed order), then hidden * inv_rms * weight, rounded once.
-      // two threads per row: each adds its half of the row's nTn partial sums (all loads in
-      // flight together where the halves are 16-byte aligned), one shuffle joins the halves;
-      // the order of the additions is fixed
-      {
+      // Normalisation of prs rows of one 128 x 128 tile of a complete band; the rows are in the
+      // slot (loaded from hidden_out by TMA).  m.aux >= 0: the first step of a run of tiles of
+      // band m.aux: 1/RMS of the band's 128 rows from the nTn partial sums of each row, kept in
+      // shared memory for the following steps of the run.  Two threads per row, each adds its
+      // half of the row's partial sums (all loads in flight together where the halves are
+      // 16-byte aligned), one shuffle joins the halves; the order of the additions is fixed.
+      if (m.aux >= 0) {
+        named_bar_sync(2, kRedThreads);  // every thread is done with the previous run's values
         const int row = ctid >> 1, half = ctid & 1;
         const int n_half = (P.nTn + 1) / 2;
         const int first = half * n_half;
         const int cnt = min(n_half, P.nTn - first);
-        const float* pr = P.ssq_part + (long long)(m.dst_y + row) * P.nTn + first;
+        const float* pr = P.ssq_part + (long long)(m.aux * kTile + row) * P.nTn + first;
         float sum = 0.f;
         if ((P.nTn & 7) == 0) {
           for (int q0 = 0; q0 < cnt; q0 += 32) {
@@ -728,31 +731,21 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
         }
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         if (half == 0) sh->inv_rms[row] = rsqrtf(sum / (float)P.N + P.eps);
+        named_bar_sync(2, kRedThreads);
       }
-      named_bar_sync(2, kRedThreads);
+      const uint32_t sbase = ring.base + slot * ring.slot_bytes;
       float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       acc_bf16x8(w, __ldg(reinterpret_cast<const uint4*>(P.weight + m.dst_x + (ctid & 15) * 8)));
-      // 8 independent 16-byte loads per thread in flight, then the arithmetic and the stores
-      constexpr int kIter = kTile * (kTile * 2 / 16) / kRedThreads;
-      uint4 hv[kIter];
-#pragma unroll
-      for (int k = 0; k < kIter; ++k) {
-        const int c = ctid + k * kRedThreads;
-        hv[k] = __ldcg(reinterpret_cast<const uint4*>(P.out + (long long)(m.dst_y + (c >> 4)) * P.N + m.dst_x + (c & 15) * 8));
-      }
-#pragma unroll
-      for (int k = 0; k < kIter; ++k) {
-        const int c = ctid + k * kRedThreads;
-        const int row = c >> 4;
+      const int n_chunks = ring.prs * (kTile * 2 / 16);
+      for (int c = ctid; c < n_chunks; c += kRedThreads) {
+        const int row = m.dst_y + (c >> 4);  // row of hidden_out; its band row is row % 128
         float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        acc_bf16x8(h, hv[k]);
-        const float inv = sh->inv_rms[row];
+        acc_bf16x8(h, ld_shared_v4(sbase + c * 16));
+        const float inv = sh->inv_rms[row & (kTile - 1)];
 #pragma unroll
         for (int e = 0; e < 8; ++e) h[e] = h[e] * inv * w[e];
-        __stcs(reinterpret_cast<uint4*>(P.norm_out + (long long)(m.dst_y + row) * P.N + m.dst_x + (c & 15) * 8),
-               pack_bf16x8(h));
+        __stcs(reinterpret_cast<uint4*>(P.norm_out + (long long)row * P.N + m.dst_x + (c & 15) * 8), pack_bf16x8(h));
       }
-      named_bar_sync(2, kRedThreads);  // inv_rms is rewritten by the next normalisation step
     }
     // one arrival per warp returns the slot (a push step is forwarded by the store warp alone;
     // the arrival then only says that this warp has read the slot's header)
@@ -810,6 +803,45 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       ok = __all_sync(0xffffffffu, free_slot);
       ring = make_ring(smem_base, 1, P, sh);
       it = 0;
+    };
+    // Layer chain: normalisation tasks (one per tile of the rank's partition, band by band) are
+    // handed out through one counter in runs of kRun tiles; a run's steps bring the rows of
+    // hidden_out into ring slots, and the band's 1/RMS values are computed once per run.
+    constexpr int kRun = 4;
+    int* const norm_head = &P.list_head[P.x];
+    // issues the steps of the run of n tiles that starts at tile i (lane 0 does the work)
+    auto issue_norm_run = [&](int i, int n) {
+      bool run_ok = true;
+      if (lane == 0) {
+        int band_seen = -1;
+        for (int t = i; run_ok && t < min(i + n, P.Q); ++t) {
+          const int band = t / P.nTn, tc = t - band * P.nTn;
+          if (band != band_seen) {
+            // (the run may reach into the next band, which may not be complete yet)
+            run_ok = wait_count(&P.band_ctr[band], (unsigned)P.nTn, P);
+            if (!run_ok) break;
+            fence_async_all();  // the TMA reads of hidden_out are ordered after the acquire
+          }
+          for (int u = 0; run_ok && u < kTile / ring.prs; ++u) {
+            const int slot = it % ring.n_slots;
+            run_ok = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+            if (!run_ok) break;
+            SlotMeta& m = sh->meta[ring.id][slot];
+            m.kind = 2;
+            m.dst_x = tc * kTile;
+            m.dst_y = band * kTile + u * ring.prs;
+            m.aux = (band != band_seen) ? band : -1;
+            band_seen = band;
+            mbar_arrive_expect_tx(ring.full(slot), ring.prs * kTile * 2);
+            tma_load_2d_hint(ring.base + slot * ring.slot_bytes, &maps.h_ld[ring.geom], tc * kTile,
+                             band * kTile + u * ring.prs, ring.full(slot), pol);
+            it += 1;
+          }
+        }
+        if (!run_ok) report(P, -ENTWINE_ERR_TIMEOUT, -7);
+      }
+      ok = __all_sync(0xffffffffu, run_ok);
+      it = __shfl_sync(0xffffffffu, it, 0);
     };
     // Drains list j.  Claims go through the list's head counter in runs of up to P.claim
     // consecutive tasks, so the list is consumed in order whoever executes it (Sec. 3.1).  This
@@ -1065,7 +1097,6 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     // waits until all nTn tiles of its band are reduced; the reducing warps read the band from
     // L2 themselves, the ring slot only hands them the task.
     if (NORM && ok && n_lists > 0) {
-      int* head = &P.list_head[P.x];
       while (ok) {
         // Wait for the band at the head of the task counter BEFORE claiming: a CTA that waits
         // holds no task, so the tasks of a band that completes are shared by every CTA that is
@@ -1073,15 +1104,10 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         int i = P.Q;
         bool band_ok = true;
         if (lane == 0) {
-          const int peek = *reinterpret_cast<volatile int*>(head);
+          const int peek = *reinterpret_cast<volatile int*>(norm_head);
           if (peek < P.Q) {
             band_ok = wait_count(&P.band_ctr[peek / P.nTn], (unsigned)P.nTn, P);
-            if (band_ok) {
-              i = atomicAdd(head, 1);
-              // the claim may belong to the next band already
-              if (i < P.Q && i / P.nTn != peek / P.nTn)
-                band_ok = wait_count(&P.band_ctr[i / P.nTn], (unsigned)P.nTn, P);
-            }
+            if (band_ok) i = atomicAdd(norm_head, kRun);
           }
         }
         ok = __all_sync(0xffffffffu, band_ok);
@@ -1091,24 +1117,9 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         }
         i = __shfl_sync(0xffffffffu, i, 0);
         if (i >= P.Q) break;
-        const int band = i / P.nTn, tc = i - band * P.nTn;
         maybe_switch();
         if (!ok) break;
-        bool free_slot = true;
-        if (lane == 0) {
-          const int slot = it % ring.n_slots;
-          free_slot = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
-          if (free_slot) {
-            SlotMeta& m = sh->meta[ring.id][slot];
-            m.kind = 2;
-            m.dst_x = tc * kTile;
-            m.dst_y = band * kTile;
-            m.aux = -1;
-            mbar_arrive(ring.full(slot));
-          }
-        }
-        ok = __all_sync(0xffffffffu, free_slot);
-        it += 1;
+        issue_norm_run(i, kRun);
       }
     }
     // end-of-work marker so that the other consumer warps leave their loops
@@ -1166,7 +1177,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         break;
       }
       if (m.kind == 0 || (NORM && (m.kind == 2 || m.kind == 3))) {
-        if (NORM && m.aux >= 0) {
+        if (NORM && m.kind == 0 && m.aux >= 0) {
           // layer chain: the last step of a reduce task counts its tile in the band
           fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
           atomicAdd(&P.band_ctr[m.aux], 1u);
@@ -2139,7 +2150,8 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
          (comm ? make_map3(&maps.p_ld[id], peers, g.W - 1, g.M, g.N, kTile, rs, g.W - 1)
                : make_map3(&maps.p_ld[id], d->C, 1, g.M, g.N, kTile, rs, 1)) &&
          make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, prs, false) &&
-         make_map(&maps.res_ld[id], norm ? norm->residual : d->C, norm ? g.R : g.M, g.N, kTile, prs, false);
+         make_map(&maps.res_ld[id], norm ? norm->residual : d->C, norm ? g.R : g.M, g.N, kTile, prs, false) &&
+         make_map(&maps.h_ld[id], norm ? out : d->C, norm ? g.R : g.M, g.N, kTile, prs, false);
   }
   if (!ok) return ENTWINE_ERR_CUDA;
   if (pair) rc = launch_bn<256, true>(p, kp, maps, grid, stream);
@@ -2285,7 +2297,8 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
          make_map3(&maps.p_hi[id], hi, std::max(W - 1 - r, 1), g.M, g.N, kTile, rs, std::max(W - 1 - r, 1),
                    stride) &&
          make_map(&maps.send_st[id], own_buf, g.M, g.N, kTile, prs, false) &&
-         make_map(&maps.res_ld[id], own_buf, g.M, g.N, kTile, prs, false);
+         make_map(&maps.res_ld[id], own_buf, g.M, g.N, kTile, prs, false) &&
+         make_map(&maps.h_ld[id], own_buf, g.M, g.N, kTile, prs, false);
   }
   if (!ok) return ENTWINE_ERR_CUDA;
   if (pair) rc = launch_bn<256, true, false, true>(p, kp, maps, grid, stream);
