@@ -1071,6 +1071,12 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     };
     // the CTA's own list first
     if (n_lists > 0) drain(first_list);
+    // consumer alone on fewer CTAs than lists: the lists without a CTA of their own are dealt out
+    // round-robin before anybody scans for leftovers (CTAs scanning in the same order would all
+    // try the same list first)
+    if (P.mode == MODE_COMM_ONLY && n_lists > 1) {
+      for (int j = first_list + (int)gridDim.x; ok && j < P.x; j += (int)gridDim.x) drain(j);
+    }
     // then the other lists: every lane looks at one list per round, lists with work are drained
     while (ok && n_lists > 1) {
       bool any = false;
