@@ -12,7 +12,12 @@
  *     memory.  The library never takes ownership of caller buffers.
  *   - No function synchronises the device unless its comment says so.
  *   - A plan is not thread-safe; calls on one plan must be issued from one thread and are
- *     serialised on the device by stream order (use one stream per plan).
+ *     serialised on the device by stream order (use one stream per plan; if the stream changes
+ *     between two calls, the new stream is made to wait for the plan's previous call).
+ *   - Launches of DIFFERENT plans must not overlap on the device either: a launch fills the
+ *     GPU with one CTA per SM whose producers and consumers wait on each other, and two
+ *     half-resident launches would each wait (boundedly: both end in ENTWINE_ERR_TIMEOUT) for
+ *     CTAs that cannot start.  Put them on one stream or order them with events.
  *
  * Notation (paper Sec. 3.1 / 4.2): R = M/W rows per output partition; reduction tile
  * 128x128; producer block 128 x BN with BN in {128,256}; cpb = BN/128; nTn = N/128;
@@ -20,8 +25,8 @@
  * emulated rank; x = number of consumer (communication) task lists.
  *
  * Data layout (all bf16, row-major, contiguous)
- *   A             [M, K_local]
- *   B             [N, K_local]   the rank's shard of the layer weight (K contiguous), so the
+ *   A             [M, K_local]   rows lda elements apart (ENTWINE_OPT_LDA, default K_local)
+ *   B             [N, K_local]   rows ldb elements apart (ENTWINE_OPT_LDB, default K_local): the rank's shard of the layer weight (K contiguous), so the
  *                                rank's partial output is C = A . B^T, [M, N]
  *   peer_partials [W-1, M, N]    incoming partial outputs of the other ranks in ascending
  *                                rank order (slot q(w) = w < r ? w : w-1).  Only rows
@@ -108,6 +113,23 @@ enum {
   ENTWINE_OPT_STAGES          = 11, /* stages of the producer's operand ring (2..6); the shared
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */
+  ENTWINE_OPT_KBLOCKS_PER_STAGE = 15, /* k-blocks (64 elements of K_local) per stage of the operand
+                                      ring: 1 or 2; 0 (default): 2 where a k-block of both operands
+                                      is 32 KiB (CTA pairs, BN = 128), else 1.  With 2 and K_local a
+                                      multiple of 64 an operand's share of a stage arrives as one
+                                      32 KiB TMA box                                                */
+  ENTWINE_OPT_LDA             = 16, /* leading dimension of A in elements (row pitch), a multiple of 8
+                                      and >= K_local; 0 (default) = K_local.  May change between
+                                      launches                                                     */
+  ENTWINE_OPT_LDB             = 17, /* the same for B                                              */
+  ENTWINE_OPT_REG_CONSUMER    = 18, /* how the consumer warps of a CTA that still produces move their
+                                      tiles.  1 (default): whole tiles through registers with plain
+                                      128-bit loads and stores, so that all shared memory and the
+                                      SM's TMA unit serve the operand ring; 0: through a small
+                                      shared-memory ring filled by TMA beside the operand stages.
+                                      Once a CTA's producer work is over (and in dedicated consumer
+                                      CTAs) tiles always go through the large TMA ring.  The layer
+                                      chain always uses the ring                                   */
   ENTWINE_OPT_COLOCATE        = 9  /* 1 (default): with TAIL_HELP (or n_comm_sms = 0) a producer
                                       CTA's consumer warps take tasks while its tensor-core work
                                       is still running, through a small shared-memory ring beside
@@ -181,7 +203,8 @@ int entwine_gemm_rs(entwine_plan_t plan, const void* A, const void* B,
                     void* stream);
 
 /*
- * entwine_gemm_rs_host - the same call for HOST buffers (same layouts): copies A, B and
+ * entwine_gemm_rs_host - the same call for HOST buffers (same layouts, always contiguous: the
+ * leading-dimension options apply to device operands only): copies A, B and
  * rows [r*R,(r+1)*R) of each peer partial to plan-owned device staging buffers, runs the
  * fused kernel, copies out_shard and send_bufs back and synchronises the plan's internal
  * stream before returning.  Pinned host memory makes the copies asynchronous with each
@@ -291,7 +314,11 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]);
  *               writes what entwine_last_status would (code, CTA, where, flags published,
  *               tiles reduced, tiles pushed, T_G ns, T_end ns) and returns the code.
  * The plan supplies the shape, order, budget and options; its own workspace is not touched
- * and entwine_last_status does not report this call.
+ * and entwine_last_status does not report this call.  With status_out == NULL nothing reports it:
+ * a device-side timeout or index failure of that call then goes unnoticed (its outputs are
+ * incomplete), so pass status_out wherever the result matters.  Options that this entry point
+ * does not implement (a release group other than 1, a withheld peer flag) make it return
+ * ENTWINE_ERR_INVALID.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
  * caches it per device: make that first call outside any stream capture.  All calls on a

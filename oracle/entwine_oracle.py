@@ -26,8 +26,10 @@ Parity status of each function (what pins it is in tests/test_oracle_*.py):
   schedule, flag_sequence          pinned: Eq. 1 closed form, the worked examples of Fig. 1
                                    and Fig. 3, the printed wave counts, bijection
   consumer_lists (reduce part)     pinned: Fig. 3 (C0 -> t0,t2,t4; C1 -> t1,t3,t5)
-  consumer_lists (push part)       parity unpinned by the paper (the paper has no push;
-                                   the rule is this build's reading, see its docstring)
+  consumer_lists (push part)       the paper has no push; the rule is this build's reading of
+                                   Sec. 3.1's assignment applied to the non-owned tiles (see
+                                   its docstring).  Pinned: hand-written lists for the Fig. 3
+                                   shape in both traversals, coverage, balance
   index_maps, traffic_counts       pinned: Eq. 2 volume, brute-force scatter on tiny shapes
   partial_gemm, reduce_scatter_ref pinned: brute-force triple loop, identity / one-hot /
                                    zero special cases, concat(shards) == unsplit GEMM
@@ -36,9 +38,9 @@ Parity status of each function (what pins it is in tests/test_oracle_*.py):
                                    the rounding bound derived in its docstring
   rmsnorm_ref, layer_chain_ref     pinned: closed forms (constant rows, one-hot rows, scale
                                    invariance at eps = 0), torch's rms_norm in float64
-  norm_task_order                  parity unpinned by the paper (the paper evaluates the
-                                   operator chain of Sec. 5.2.3 but does not fuse it; the
-                                   band rule is this build's design, see its docstring)
+  norm_task_order                  the paper evaluates the operator chain of Sec. 5.2.3 but does
+                                   not fuse it; the band rule is this build's design (see its
+                                   docstring).  Pinned: a hand-listed 2-band x 3-column case
 """
 from __future__ import annotations
 
@@ -454,20 +456,3 @@ def gemm_rs(A_bits, B_bits, peers_bits, r: int, W: int, BN: int, order: int, x: 
         out.update(C_rows=partial_gemm(A_bits[rows], B_bits),
                    S_rows=abs_gemm(A_bits[rows], B_bits))
     return out
-
-
-def valid_completion_log(log, P_blk: int, G: int) -> bool:
-    """A physical completion log (block positions in the order they finished) is valid iff
-    it is a permutation of [0, P_blk) in which the blocks of each persistent producer
-    (p congruent to g modulo G) appear in increasing order (Sec. 3.1: the mapping fixes
-    the logical order only)."""
-    log = [int(v) for v in log]
-    if sorted(log) != list(range(P_blk)):
-        return False
-    last = {}
-    for p in log:
-        g = p % G
-        if g in last and last[g] > p:
-            return False
-        last[g] = p
-    return True

@@ -9,6 +9,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "entwine_internal.h"
 
@@ -18,7 +19,8 @@ namespace entwine {
 // compile-time shape of the kernel
 // ------------------------------------------------------------------------------------------
 constexpr int kBM = 128;          // producer block rows = reduction tile rows
-constexpr int kBK = 64;           // K elements per pipeline stage (128 bytes = one swizzle row)
+constexpr int kBK = 64;           // K elements per k-block (128 bytes = one swizzle row); a pipeline
+                                  // stage holds P.kpb k-blocks of both operands
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit operands
 // Warp roles of the 16 warps of a CTA.  Producer work (warps 0, 1, 4-7) and consumer work
 // (warps 2, 3, 8-15) run side by side in a producer CTA: the tensor pipe is driven by one
@@ -52,6 +54,7 @@ constexpr int kStagingBytes = 2 * kEpiBufBytes;
 constexpr int kRingBOff = 0;
 constexpr int kRingBBytes = 196608;
 constexpr int kMaxSlots = 8;
+constexpr int kRegSlots = 4;       // task descriptors in flight between the claiming and the reducing warps
 constexpr int kMaxStages = 6;
 constexpr int kBarOff = kDataBytes;
 constexpr int kBarBytes = 640;
@@ -70,9 +73,9 @@ template <int BN, bool PAIR>
 struct Cfg {
   static_assert(!PAIR || BN == 256, "pair tiles are 256 wide");
   static constexpr int kBRows = PAIR ? 128 : BN;  // rows of B this CTA loads per stage
-  static constexpr int kABytes = kBM * kBK * 2;
-  static constexpr int kBBytes = kBRows * kBK * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kABytes = kBM * kBK * 2;     // one k-block of A
+  static constexpr int kBBytes = kBRows * kBK * 2;  // one k-block of this CTA's rows of B
+  static constexpr int kKBlockBytes = kABytes + kBBytes;  // a stage is P.kpb of these: all of A, then all of B
   static constexpr int kTmemCols = 2 * BN;  // two accumulators: epilogue overlaps next mainloop
 };
 
@@ -91,11 +94,18 @@ struct KParams {
   int prefetch;   // pull the next reduce task's peer tiles into L2 ahead of its loads
   int l2_hints;   // consumer TMA traffic carries an evict-first L2 policy
   int stages;     // operand-ring stages of the producer
+  int kpb;        // k-blocks (64 elements of K) per stage
+  int k3d;        // 1: a stage's k-blocks of one operand arrive as ONE 3-D TMA box (the SM's TMA unit keeps
+                  // only about two load instructions in flight, so bytes per instruction bound its rate)
   int ring_a_off, ring_a_bytes;  // consumer ring A (after the epilogue staging)
   int stage_area;                // bytes of the operand stages
   int early_b;                   // 1: a producer CTA's ring B is its operand stages, used as soon as its
                                  // last MMA has completed; 0: the full ring B once its producer work is over
   int ring_a_geom;               // which geometry ring A uses (0: 16 KiB steps, 1: 32 KiB steps)
+  int reg_a;      // 1: while a producer CTA still produces, its consumer warps run whole-tile tasks from
+                  // registers (plain loads and stores) instead of a shared-memory ring: ring A then holds
+                  // task descriptors only, all shared memory goes to the operand stages, and the SM's TMA
+                  // unit serves the operand loads alone
   int skip_wait;  // treat every flag as published (consumer in isolation)
   int claim;      // most consecutive tasks taken from a list per claim
   int release_group;     // blocks released together (1 = each block by itself; -1, -2: see the header)
@@ -109,6 +119,10 @@ struct KParams {
   unsigned long long wait_budget_ns;
   // memory
   __nv_bfloat16* out;            // out_shard [R][N] (written by the reducing warps)
+  const __nv_bfloat16* cws;      // the rank's partial C [M][N] as the consumer reads it (register path)
+  const __nv_bfloat16* peers;    // incoming partials [W-1][M][N] (register path; pull mode: see heap)
+  __nv_bfloat16* send;           // send_bufs [W-1][R][N] (register path)
+  long long heap_buf_off;        // pull mode: offset of this call's partial-output buffer inside a segment
   unsigned* flags_own;           // [W][Q]
   const unsigned* flags_peer;    // [W-1][Q]
   const Task* tasks;
@@ -136,7 +150,8 @@ struct KParams {
 // Tensor maps of one launch.  Loads of A and B and the epilogue's stores of C use the
 // 128-byte swizzle; the consumer's maps are plain row-major boxes of 128 columns x rs rows.
 struct KMaps {
-  CUtensorMap a, b;      // operands
+  CUtensorMap a, b;      // operands, one k-block per box
+  CUtensorMap a3, b3;    // operands viewed as [K/64][rows][64]: one box brings kpb k-blocks (k3d)
   CUtensorMap c_st;      // partial C, box 64 x 128, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
@@ -284,6 +299,14 @@ __device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtens
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
       ".L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair_hint(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                                      uint32_t bar_cluster_addr, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      ".L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar_cluster_addr), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
@@ -477,7 +500,8 @@ __device__ __forceinline__ int pair_position(const KParams& P, int u, int rank) 
 // ------------------------------------------------------------------------------------------
 struct SlotMeta {
   int kind;      // 0 reduce step, 1 push step, 2 normalisation of a tile, 3 residual rows of the tile whose
-                 // reduce steps follow, -1 end of work, -2 continue on ring B
+                 // reduce steps follow, 4 / 5 whole reduce / push task done from registers (dst_y: first
+                 // destination row, aux: first row in the [M,N] buffers), -1 end of work, -2 continue on ring B
   int dst_x;     // column of the destination box
   int dst_y;     // row of the destination box in the destination buffer
   int aux;       // layer chain: band (tile row) whose count the last step of a reduce task raises, else -1
@@ -600,13 +624,108 @@ __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KPar
   r.slot_bytes = P.slot_bytes[r.geom];
   r.sub_bytes = r.rs * kTile * 2;
   r.n_slots = min(kMaxSlots, (id == 0 ? P.ring_a_bytes : sh->ring_b_bytes) / r.slot_bytes);
+  if (id == 0 && P.reg_a) r.n_slots = kRegSlots;  // descriptors only
   return r;
+}
+
+// ------------------------------------------------------------------------------------------
+// Whole-tile tasks from registers (the consumer warps of a CTA that still produces).  256 threads
+// share a 128 x 128 tile: thread ctid takes the 16-byte chunks ctid, ctid + 256, ... (row c / 16,
+// column chunk c % 16), so a warp's load covers two 256-byte row segments.  Up to 16 loads of 16
+// bytes are in flight per thread.  The partial C was written through the async proxy by other
+// SMs and is read at L2 (never from this SM's L1); the flags were acquired by the claiming warp,
+// whose barrier arrival orders these loads after them.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_l2_v4(const __nv_bfloat16* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ld_stream_v4(const __nv_bfloat16* p) {
+  uint4 v;
+  asm volatile("ld.global.cs.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+// contribution of peer slot q (ascending rank order with the own rank left out), as [M][N]
+template <bool PULL>
+__device__ __forceinline__ const __nv_bfloat16* peer_base(const KParams& P, int q) {
+  if (PULL) {
+    const int w = q + (q >= P.r ? 1 : 0);
+    return reinterpret_cast<const __nv_bfloat16*>(P.heap + (long long)w * P.heap_stride + P.heap_buf_off);
+  }
+  return P.peers + (long long)q * P.M * P.N;
+}
+template <int WW, bool PULL>
+__device__ __forceinline__ void reg_reduce_tile(const KParams& P, int ctid, int col, int src_row, int dst_row) {
+  constexpr int kChunks = kTile * (kTile * 2 / 16) / kRedThreads;  // 8 per thread
+  constexpr int NB = (16 / WW) < 1 ? 1 : ((16 / WW) > kChunks ? kChunks : (16 / WW));
+  const long long N = P.N;
+#pragma unroll 1
+  for (int i0 = 0; i0 < kChunks; i0 += NB) {
+    uint4 v[NB][WW];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const int c = ctid + (i0 + b) * kRedThreads;
+      const long long off = (long long)(src_row + (c >> 4)) * N + col + (c & 15) * 8;
+      v[b][0] = ld_l2_v4(P.cws + off);
+#pragma unroll
+      for (int q = 1; q < WW; ++q) v[b][q] = ld_stream_v4(peer_base<PULL>(P, q - 1) + off);
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      const int c = ctid + (i0 + b) * kRedThreads;
+      // local contribution first, then the peers in ascending rank order, fp32, one rounding
+      float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int q = 0; q < WW; ++q) acc_bf16x8(a, v[b][q]);
+      __stcs(reinterpret_cast<uint4*>(P.out + (long long)(dst_row + (c >> 4)) * N + col + (c & 15) * 8), pack_bf16x8(a));
+    }
+  }
+}
+// any W: chunk by chunk, the peers' loads of a chunk in flight four at a time
+template <bool PULL>
+__device__ __forceinline__ void reg_reduce_tile_any(const KParams& P, int ctid, int col, int src_row, int dst_row) {
+  constexpr int kChunks = kTile * (kTile * 2 / 16) / kRedThreads;
+  const long long N = P.N;
+#pragma unroll 1
+  for (int i = 0; i < kChunks; ++i) {
+    const int c = ctid + i * kRedThreads;
+    const long long off = (long long)(src_row + (c >> 4)) * N + col + (c & 15) * 8;
+    float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    acc_bf16x8(a, ld_l2_v4(P.cws + off));
+#pragma unroll 1
+    for (int q0 = 0; q0 < P.W - 1; q0 += 4) {
+      uint4 v[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        v[j] = (q0 + j < P.W - 1) ? ld_stream_v4(peer_base<PULL>(P, q0 + j) + off) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (q0 + j < P.W - 1) acc_bf16x8(a, v[j]);
+    }
+    __stcs(reinterpret_cast<uint4*>(P.out + (long long)(dst_row + (c >> 4)) * N + col + (c & 15) * 8), pack_bf16x8(a));
+  }
+}
+__device__ __forceinline__ void reg_push_tile(const KParams& P, int ctid, int col, int src_row, int dst_row) {
+  constexpr int kChunks = kTile * (kTile * 2 / 16) / kRedThreads;
+  const long long N = P.N;
+  uint4 v[kChunks];
+#pragma unroll
+  for (int i = 0; i < kChunks; ++i) {
+    const int c = ctid + i * kRedThreads;
+    v[i] = ld_l2_v4(P.cws + (long long)(src_row + (c >> 4)) * N + col + (c & 15) * 8);
+  }
+#pragma unroll
+  for (int i = 0; i < kChunks; ++i) {
+    const int c = ctid + i * kRedThreads;
+    __stcs(reinterpret_cast<uint4*>(P.send + (long long)(dst_row + (c >> 4)) * N + col + (c & 15) * 8), v[i]);
+  }
 }
 
 // The reducing warps' loop (Sec. 4.2, ReduceTile).  NORM selects the layer-chain variant, which
 // carries the tile's residual in registers and handles the residual and normalisation steps; the
 // plain variant is compiled without any of that state.
-template <bool NORM>
+template <bool NORM, bool PULL>
 __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, uint32_t smem_base, Ring ring) {
   const int lane = threadIdx.x & 31;
   const int ctid = threadIdx.x - kRedWarp0 * 32;
@@ -635,7 +754,15 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
       ph = 0;
       continue;
     }
-    if (!NORM && m.kind == 0) {
+    if (!NORM && m.kind == 4) {
+      // a whole reduce task from registers (ReduceTile of Sec. 4.2 on all 128 rows of the tile)
+      if (P.W == 2) reg_reduce_tile<2, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
+      else if (P.W == 4) reg_reduce_tile<4, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
+      else if (P.W == 8) reg_reduce_tile<8, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
+      else reg_reduce_tile_any<PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
+    } else if (!NORM && !PULL && m.kind == 5) {
+      reg_push_tile(P, ctid, m.dst_x, m.aux, m.dst_y);
+    } else if (!NORM && m.kind == 0) {
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
       const int rs = ring.rs, sub_bytes = ring.sub_bytes;
       __nv_bfloat16* dst = P.out + (long long)m.dst_y * P.N + m.dst_x;
@@ -788,7 +915,8 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         // Otherwise ring B's last slots overlap ring A's memory, and every ring-A step in flight
         // must have returned its slot first: slot s has been used uses(s) times; its last use,
         // number uses(s) - 1, is over when its empty barrier completes the phase of that parity.
-        for (int sl = 0; !P.early_b && free_slot && sl < ring.n_slots; ++sl) {
+        // (In register mode ring A holds no data at all.)
+        for (int sl = 0; !P.early_b && !P.reg_a && free_slot && sl < ring.n_slots; ++sl) {
           const int uses = (it - sl + ring.n_slots - 1) / ring.n_slots;
           if (uses > 0) free_slot = mbar_wait(ring.empty(sl), (uses - 1) & 1, P, sh);
         }
@@ -999,6 +1127,29 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           }
           maybe_switch();
           if (!ok) break;
+          if (!NORM && ring.id == 0 && P.reg_a) {
+            // register path: the reducing warps load the tile themselves; one descriptor per task
+            bool slot_ok = true;
+            if (lane == 0) {
+              const int slot = it % ring.n_slots;
+              slot_ok = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+              if (slot_ok) {
+                SlotMeta& m = sh->meta[0][slot];
+                m.kind = 4 + kind;
+                m.dst_x = col;
+                m.dst_y = dst_row;
+                m.aux = src_row;
+                mbar_arrive(ring.full(slot));
+                if (kind == 0) cnt->reduced++;
+                else cnt->pushed++;
+              } else {
+                report(P, -ENTWINE_ERR_TIMEOUT, base + i);
+              }
+            }
+            ok = __all_sync(0xffffffffu, slot_ok);
+            it += 1;
+            continue;
+          }
           const int rows = kind == 0 ? ring.rs : ring.prs;  // rows of the tile per ring step
           const int n_steps = kTile / rows;
           bool steps_ok = true;
@@ -1139,7 +1290,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     __syncwarp();
   } else if (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32) {
     // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
-    reducer_role<NORM>(P, sh, smem_base, ring);
+    reducer_role<NORM, PULL>(P, sh, smem_base, ring);
   } else if (warp == kStoreWarp && lane == 0) {
     // ---------------- forward push slots with TMA stores, recycle all slots ----------------
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
@@ -1182,7 +1333,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         sh->abort = 1;
         break;
       }
-      if (m.kind == 0 || (NORM && (m.kind == 2 || m.kind == 3))) {
+      if (m.kind == 0 || m.kind >= 4 || (NORM && (m.kind == 2 || m.kind == 3))) {
         if (NORM && m.kind == 0 && m.aux >= 0) {
           // layer chain: the last step of a reduce task counts its tile in the band
           fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
@@ -1251,6 +1402,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * kMaxStages + 2 + a); };
   const int n_stages = P.stages;
+  const int stage_bytes = P.kpb * C::kKBlockBytes;
   const uint32_t tmem_slot = smem_base + kBarOff + kBarTmemSlot;
   const uint32_t pair_bar = smem_base + kBarOff + kBarPair;
   auto staged_bar = [&](int b) { return smem_base + kBarOff + kBarStaging + 8u * b; };
@@ -1354,20 +1506,42 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         int d, l;
         block_of(i, &d, &l);
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
-        for (int kb = 0; kb < KB; ++kb) {
+        const int b_row = nb * BN + (PAIR ? (int)cta_rank * C::kBRows : 0);
+        for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1, P, &sh)) { ok = false; break; }
-          const uint32_t a_dst = smem_base + stage * C::kStageBytes;
-          if (PAIR) {
-            // both CTAs' bytes are counted on the leader's barrier, which the leader arms
-            if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * C::kStageBytes);
-            const uint32_t lead_bar = map_to_cta(full_bar(stage), 0);
-            tma_load_2d_pair_hint(a_dst, &maps.a, kb * kBK, mb * kBM, lead_bar, op_pol);
-            tma_load_2d_pair_hint(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN + (int)cta_rank * C::kBRows,
-                                  lead_bar, op_pol);
+          const uint32_t a_dst = smem_base + stage * stage_bytes;
+          const uint32_t b_dst = a_dst + P.kpb * C::kABytes;
+          // k-blocks of this stage that exist (a ragged last stage is filled, and multiplied, in part)
+          const int nkb = min(P.kpb, KB - kb0);
+          const uint32_t lead_bar = PAIR ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
+          if (P.k3d) {
+            // one box per operand: [kpb k-blocks][rows][64]; k-blocks past the end of K read as zero
+            if (PAIR) {
+              // both CTAs' bytes are counted on the leader's barrier, which the leader arms
+              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * stage_bytes);
+              tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
+              tma_load_3d_pair_hint(b_dst, &maps.b3, 0, b_row, kb0, lead_bar, op_pol);
+            } else {
+              mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
+              tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, full_bar(stage), op_pol);
+              tma_load_3d_hint(b_dst, &maps.b3, 0, b_row, kb0, full_bar(stage), op_pol);
+            }
           } else {
-            mbar_arrive_expect_tx(full_bar(stage), C::kStageBytes);
-            tma_load_2d_hint(a_dst, &maps.a, kb * kBK, mb * kBM, full_bar(stage), op_pol);
-            tma_load_2d_hint(a_dst + C::kABytes, &maps.b, kb * kBK, nb * BN, full_bar(stage), op_pol);
+            if (PAIR) {
+              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * nkb * C::kKBlockBytes);
+            } else {
+              mbar_arrive_expect_tx(full_bar(stage), nkb * C::kKBlockBytes);
+            }
+            for (int kk = 0; kk < nkb; ++kk) {
+              const int kx = (kb0 + kk) * kBK;
+              if (PAIR) {
+                tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, lead_bar, op_pol);
+                tma_load_2d_pair_hint(b_dst + kk * C::kBBytes, &maps.b, kx, b_row, lead_bar, op_pol);
+              } else {
+                tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, full_bar(stage), op_pol);
+                tma_load_2d_hint(b_dst + kk * C::kBBytes, &maps.b, kx, b_row, full_bar(stage), op_pol);
+              }
+            }
           }
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
@@ -1385,17 +1559,21 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
           if (!mbar_wait(full_bar(stage), phase, P, &sh)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_s = smem_base + stage * C::kStageBytes;
-          const uint64_t a_desc = smem_desc_sw128(a_s);
-          const uint64_t b_desc = smem_desc_sw128(a_s + C::kABytes);
+          const uint32_t a_s = smem_base + stage * stage_bytes;
+          const uint32_t b_s = a_s + P.kpb * C::kABytes;
+          const int nkb = min(P.kpb, KB - kb0);
+          for (int kk = 0; kk < nkb; ++kk) {
+            const uint64_t a_desc = smem_desc_sw128(a_s + kk * C::kABytes);
+            const uint64_t b_desc = smem_desc_sw128(b_s + kk * C::kBBytes);
 #pragma unroll
-          for (int k = 0; k < kBK / kUmmaK; ++k) {
-            // advancing K by 16 elements = 32 bytes = 2 descriptor address units
-            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-            else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              // advancing K by 16 elements = 32 bytes = 2 descriptor address units
+              if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb0 | kk | k) != 0);
+              else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb0 | kk | k) != 0);
+            }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if (PAIR) tc_commit_pair(empty_bar(stage));
@@ -1413,7 +1591,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       //      128 rows x 64 columns through two staging buffers; the publishing warp stores them,
       //      so these warps never wait for global memory ----
       const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
-      const uint32_t stg0 = smem_base + n_stages * C::kStageBytes + (q * 32 + lane) * 128;
+      const uint32_t stg0 = smem_base + n_stages * stage_bytes + (q * 32 + lane) * 128;
       int acc = 0;
       uint32_t acc_phase = 0;
       int nbox = 0;  // boxes staged so far: buffer nbox & 1, use (nbox >> 1)
@@ -1501,7 +1679,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           }
           if (!mbar_wait(staged_bar(buf), (nbox >> 1) & 1, P, &sh)) { ok = false; break; }
           tma_store_2d(&maps.c_st, nb * BN + j * 64, mb * kBM,
-                       smem_base + n_stages * C::kStageBytes + buf * kEpiBufBytes);
+                       smem_base + n_stages * stage_bytes + buf * kEpiBufBytes);
           bulk_commit();
           bulk_wait_read<1>();  // the stores before this one have read their buffers
           free_upto(nbox - 1);
@@ -1692,6 +1870,7 @@ struct DeviceState {
   bool captured = false;  // a launch of this plan has been captured into a CUDA graph
   bool status_pending = false;
   cudaStream_t last_stream = nullptr;
+  cudaEvent_t switch_event = nullptr;  // orders a new stream after the plan's last launch
   int64_t withheld = -1;
   // staging for the host-buffer entry point
   cudaStream_t own_stream = nullptr;
@@ -1728,11 +1907,11 @@ static EncodeTiledFn get_encode_fn() {
 // out-of-range elements read as zero (K tails).  `swizzle128` selects the 128-byte swizzle
 // (box_cols must then be 64 elements = 128 bytes).
 static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_cols,
-                     int box_rows, bool swizzle128) {
+                     int box_rows, bool swizzle128, int64_t pitch_elems = 0) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
-  cuuint64_t strides[1] = {cuuint64_t(cols) * 2};
+  cuuint64_t strides[1] = {cuuint64_t(pitch_elems > 0 ? pitch_elems : cols) * 2};
   cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
   cuuint32_t estr[2] = {1, 1};
   CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
@@ -1756,6 +1935,37 @@ static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_
                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return rc == CUDA_SUCCESS;
+}
+
+// Operand maps of the producer.  a / b: one k-block (64 elements of K, 128-byte swizzle) per box.
+// a3 / b3: the same matrix seen as [K/64][rows][64] (k-blocks 128 bytes apart inside a row), so that
+// one box of kpb k-blocks fills a whole pipeline stage of that operand with one TMA instruction;
+// only where K is a multiple of 64 (the view has no partial k-block).  Returns false on an
+// encoding failure; *k3d tells whether the 3-D maps are usable.
+static bool make_operand_maps(KMaps* maps, const void* A, const void* B, const Geometry& g, int b_rows, int kpb,
+                              int64_t lda, int64_t ldb, int* k3d) {
+  *k3d = 0;
+  if (!make_map(&maps->a, A, g.M, g.K, kBK, kBM, true, lda) || !make_map(&maps->b, B, g.N, g.K, kBK, b_rows, true, ldb))
+    return false;
+  if (kpb < 2 || g.K % kBK != 0) return true;
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  bool ok = true;
+  for (int op = 0; op < 2; ++op) {
+    const int64_t rows = op == 0 ? g.M : g.N;
+    const int64_t ld = op == 0 ? (lda > 0 ? lda : g.K) : (ldb > 0 ? ldb : g.K);
+    cuuint64_t dims[3] = {cuuint64_t(kBK), cuuint64_t(rows), cuuint64_t(g.K / kBK)};
+    cuuint64_t strides[2] = {cuuint64_t(ld) * 2, cuuint64_t(kBK) * 2};
+    cuuint32_t box[3] = {cuuint32_t(kBK), cuuint32_t(op == 0 ? kBM : b_rows), cuuint32_t(kpb)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult rc = fn(op == 0 ? &maps->a3 : &maps->b3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                     const_cast<void*>(op == 0 ? A : B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    ok = ok && rc == CUDA_SUCCESS;
+  }
+  *k3d = ok ? 1 : 0;  // without them a stage is filled k-block by k-block
+  return true;
 }
 
 // Tasks per claim: as many as have their flags (W per reduce task) in the 64 flag values the
@@ -1862,6 +2072,7 @@ void device_release(Plan* p) {
     cudaStreamSynchronize(d->own_stream);
     cudaStreamDestroy(d->own_stream);
   }
+  if (d->switch_event) cudaEventDestroy(d->switch_event);
   cudaFree(d->C);
   cudaFree(d->flags_own);
   cudaFree(d->flags_peer);
@@ -1884,14 +2095,28 @@ void device_release(Plan* p) {
   p->dev = nullptr;
 }
 
+// The caller moved the plan to another stream: the new stream waits, on the device, for what the
+// old one still has to do for this plan (one workspace: calls of a plan never overlap).
+static cudaError_t order_after_last_launch(DeviceState* d, cudaStream_t stream) {
+  if (!d->switch_event) {
+    cudaError_t e = cudaEventCreateWithFlags(&d->switch_event, cudaEventDisableTiming);
+    if (e != cudaSuccess) return e;
+  }
+  cudaError_t e = cudaEventRecord(d->switch_event, d->last_stream);
+  if (e != cudaSuccess) return e;
+  return cudaStreamWaitEvent(stream, d->switch_event, 0);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int BN, bool PAIR, bool NORM = false, bool PULL = false>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
   if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false>(p, kp, maps, grid, stream);
-  // per device: the shared-memory opt-in has been set, and how many clusters fit at once
+  // per device: the shared-memory opt-in has been set, and how many clusters fit at once (shared by
+  // all plans, which may be used from different threads)
   static int max_clusters[64] = {0};
   static bool configured[64] = {false};
+  static std::mutex config_mutex;
   int dev = 0;
   CK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ENTWINE_ERR_RESOURCES;
@@ -1909,6 +2134,7 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  std::lock_guard<std::mutex> lock(config_mutex);
   if (!configured[dev]) {
     CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
     int per_sm = 0;
@@ -1929,7 +2155,7 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
 // contributions (at most 16 KiB with geometry 0, 32 KiB with geometry 1), a push step moves as
 // many rows of one tile as fit in a slot.  The producer's operand ring gets `stages` stages;
 // what remains after the epilogue staging is the co-located consumer ring A.
-static int ring_geometry(const Plan* p, KParams* kp) {
+static int ring_geometry(const Plan* p, KParams* kp, bool reg_a) {
   const Geometry& g = p->g;
   for (int id = 0; id < 2; ++id) {
     const int budget = id == 0 ? 16384 : 32768;
@@ -1945,30 +2171,46 @@ static int ring_geometry(const Plan* p, KParams* kp) {
     kp->prs[id] = prs;
     kp->slot_bytes[id] = slot_bytes;
   }
-  const int stage_bytes = kBM * kBK * 2 + (p->pair ? 128 : g.BN) * kBK * 2;
+  // k-blocks per stage: two where a k-block of both operands is 32 KiB (pair tiles, 128-wide blocks), so
+  // that an operand's share of a stage is one 32 KiB TMA box
+  const int kblock_bytes = kBM * kBK * 2 + (p->pair ? 128 : g.BN) * kBK * 2;
+  int kpb = p->kpb;
+  if (kpb <= 0) {
+    kpb = (kblock_bytes <= 32768 && g.K >= 2 * kBK) ? 2 : 1;
+    // a requested number of stages that only fits with single k-blocks gets single k-blocks
+    if (kpb == 2 && p->stages > 0 && p->stages * 2 * kblock_bytes + kStagingBytes > kDataBytes) kpb = 1;
+  }
+  if (kpb * kblock_bytes > 65536) return ENTWINE_ERR_INVALID;
+  const int stage_bytes = kpb * kblock_bytes;
   int stages = p->stages;
   if (stages <= 0) {
-    // default: deep operand ring; shapes whose communication outweighs their tensor work give
-    // one stage to the co-located consumer ring
-    stages = (kDataBytes - kStagingBytes - 2 * kp->slot_bytes[0]) / stage_bytes;
-    if (stages > 5) stages = 5;
+    // default: as deep an operand ring as leaves two small slots to the co-located consumer ring;
+    // shapes whose communication outweighs their tensor work give one stage to that ring
+    stages = (kDataBytes - kStagingBytes - (reg_a ? 0 : 2 * kp->slot_bytes[0])) / stage_bytes;
+    if (stages > (reg_a ? kMaxStages : 5)) stages = reg_a ? kMaxStages : 5;
+    // rough peaks, only to rank the two kinds of work of a shape against each other
     const double t_tc = 2.0 * g.M * g.N * g.K / 1.6e15;
     const double t_hbm = double(g.M) * g.N * 2.0 * (3 * g.W - 1) / g.W / 6.5e12;
-    if (p->colocate && t_hbm > 0.5 * t_tc && stages > 3) stages -= 1;
+    if (!reg_a && p->colocate && t_hbm > 0.5 * t_tc && stages * kpb > 3) stages -= 1;
     // communication-bound shapes (K_local of a few hundred): one more stage goes to the ring
-    if (p->colocate && t_hbm > t_tc && stages > 3) stages -= 1;
+    if (!reg_a && p->colocate && t_hbm > t_tc && stages * kpb > 3) stages -= 1;
+    if (stages < 2) stages = 2;
   }
-  if (stages < 2 || stages > kMaxStages) return ENTWINE_ERR_INVALID;
+  if (stages < 2 || stages > kMaxStages || stages * stage_bytes + kStagingBytes > kDataBytes) return ENTWINE_ERR_INVALID;
   const int ring_a_off = stages * stage_bytes + kStagingBytes;
   const int ring_a_bytes = kDataBytes - ring_a_off;
-  if (ring_a_bytes < 2 * kp->slot_bytes[0]) return ENTWINE_ERR_RESOURCES;
   kp->stages = stages;
+  kp->kpb = kpb;
   kp->ring_a_off = ring_a_off;
   kp->stage_area = std::min(stages * stage_bytes, kRingBBytes);
   // ring B in the operand stages alone needs room for at least four slots to keep the tail's rate
   kp->early_b = kp->stage_area >= 4 * kp->slot_bytes[1] ? 1 : 0;
   kp->ring_a_bytes = ring_a_bytes;
   kp->ring_a_geom = ring_a_bytes >= 2 * kp->slot_bytes[1] ? 1 : 0;
+  // no room for a ring beside the operand stages: the consumer warps of a producer CTA start when
+  // its stages are free
+  kp->colocate = (p->colocate && (reg_a || ring_a_bytes >= 2 * kp->slot_bytes[0])) ? 1 : 0;
+  kp->reg_a = reg_a ? 1 : 0;
   return ENTWINE_OK;
 }
 
@@ -2033,7 +2275,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
 
   // serialise with the plan's previous launch if the caller switched streams (a graph's
   // launches are ordered by whoever replays it)
-  if (d->last_stream != stream && p->launched && !capturing) CK(cudaStreamSynchronize(d->last_stream));
+  if (d->last_stream != stream && p->launched && !capturing) CK(order_after_last_launch(d, stream));
 
   if (mode != MODE_COMM_ONLY) {
     d->epoch += 1;
@@ -2097,12 +2339,14 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  rc = ring_geometry(p, &kp);
+  rc = ring_geometry(p, &kp, p->reg_consumer && !norm);
   if (rc != ENTWINE_OK) return rc;
-  kp.colocate = p->colocate;
   kp.prefetch = p->prefetch;
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out);
+  kp.cws = (mode == MODE_COMM_ONLY && partial) ? static_cast<const __nv_bfloat16*>(partial) : d->C;
+  kp.peers = static_cast<const __nv_bfloat16*>(peers);
+  kp.send = static_cast<__nv_bfloat16*>(send);
   kp.flags_own = d->flags_own;
   kp.flags_peer = d->flags_peer;
   kp.tasks = d->tasks;
@@ -2142,11 +2386,10 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   const void* a_p = (mode != MODE_COMM_ONLY) ? A : d->C;
   const void* b_p = (mode != MODE_COMM_ONLY) ? B : d->C;
   const bool comm = mode != MODE_GEMM_ONLY;
-  bool ok = make_map(&maps.a, a_p, (mode != MODE_COMM_ONLY) ? g.M : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
-                     kBK, kBM, true) &&
-            make_map(&maps.b, b_p, (mode != MODE_COMM_ONLY) ? g.N : g.M, (mode != MODE_COMM_ONLY) ? g.K : g.N,
-                     kBK, (mode != MODE_COMM_ONLY) ? (pair ? 128 : g.BN) : kBM, true) &&
-            make_map(&maps.c_st, d->C, g.M, g.N, 64, kBM, true) &&
+  bool ok = (mode != MODE_COMM_ONLY)
+                ? make_operand_maps(&maps, a_p, b_p, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d)
+                : (make_map(&maps.a, a_p, g.M, g.N, kBK, kBM, true) && make_map(&maps.b, b_p, g.M, g.N, kBK, kBM, true));
+  ok = ok && make_map(&maps.c_st, d->C, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
@@ -2221,7 +2464,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
       return ENTWINE_ERR_CUDA;
     }
   }
-  if (d->last_stream != stream && p->launched) CK(cudaStreamSynchronize(d->last_stream));
+  if (d->last_stream != stream && p->launched) CK(order_after_last_launch(d, stream));
   if (d->captured) {
     // (the plan's own flags are not used here; heads and status are)
     const int n_heads = 2 * (p->x + 1);
@@ -2250,12 +2493,13 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  rc = ring_geometry(p, &kp);
+  rc = ring_geometry(p, &kp, p->reg_consumer != 0);
   if (rc != ENTWINE_OK) return rc;
-  kp.colocate = p->colocate;
   kp.prefetch = 0;
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out);
+  kp.cws = reinterpret_cast<const __nv_bfloat16*>(own_seg + buf_off);
+  kp.heap_buf_off = buf_off;
   kp.heap = seg0;
   kp.heap_stride = stride;
   kp.heap_flags_off = heap_flags_offset(g);
@@ -2286,8 +2530,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   std::memset(&maps, 0, sizeof(maps));
   void* own_buf = own_seg + buf_off;
   const int r = p->rank, W = g.W;
-  bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
-            make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
+  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d) &&
             make_map(&maps.c_st, own_buf, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, own_buf, g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
@@ -2440,7 +2683,14 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, cons
     CK(cudaMemcpyAsync(reinterpret_cast<char*>(d->sPeers) + off, static_cast<const char*>(peer_partials) + off,
                        part, cudaMemcpyHostToDevice, s));
   }
-  rc = launch(plan, MODE_FUSED, d->sA, d->sB, nullptr, d->sPeers, d->sOut, d->sSend, 0, s);
+  {
+    // the staging copies are contiguous whatever the leading dimensions of device operands are
+    const int64_t lda = plan->lda, ldb = plan->ldb;
+    plan->lda = plan->ldb = 0;
+    rc = launch(plan, MODE_FUSED, d->sA, d->sB, nullptr, d->sPeers, d->sOut, d->sSend, 0, s);
+    plan->lda = lda;
+    plan->ldb = ldb;
+  }
   if (rc != ENTWINE_OK) return rc;
   CK(cudaMemcpyAsync(out_shard, d->sOut, szO, cudaMemcpyDeviceToHost, s));
   CK(cudaMemcpyAsync(send_bufs, d->sSend, szS, cudaMemcpyDeviceToHost, s));
@@ -2496,7 +2746,13 @@ int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B
   // the kernel: after its inputs are up and the copies down that last read this set's results
   CK(cudaStreamWaitEvent(hp->comp, hp->up_done[s], 0));
   CK(cudaStreamWaitEvent(hp->comp, hp->d_done[s], 0));
-  rc = launch(plan, MODE_FUSED, hp->A[s], hp->B[s], nullptr, hp->peers[s], hp->out[s], hp->send[s], 0, hp->comp);
+  {
+    const int64_t lda = plan->lda, ldb = plan->ldb;
+    plan->lda = plan->ldb = 0;
+    rc = launch(plan, MODE_FUSED, hp->A[s], hp->B[s], nullptr, hp->peers[s], hp->out[s], hp->send[s], 0, hp->comp);
+    plan->lda = lda;
+    plan->ldb = ldb;
+  }
   if (rc != ENTWINE_OK) return rc;
   CK(cudaEventRecord(hp->k_done[s], hp->comp));
   CK(cudaStreamWaitEvent(hp->down, hp->k_done[s], 0));
@@ -2553,6 +2809,8 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   const Geometry& g = p->g;
   const HostTables& t = p->tables;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+  // options this entry point does not implement are refused, not ignored
+  if (p->release_group != 1 || p->withhold_peer >= 0) return ENTWINE_ERR_INVALID;
 
   // ---- sizes against the static maximum ----
   const size_t c_bytes = size_t(g.M) * g.N * 2;
@@ -2621,10 +2879,12 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.seq = 0;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
   {
-    const int grc = ring_geometry(p, &kp);
+    const int grc = ring_geometry(p, &kp, p->reg_consumer != 0);
     if (grc != ENTWINE_OK) return grc;
   }
-  kp.colocate = p->colocate;
+  kp.cws = reinterpret_cast<const __nv_bfloat16*>(base);
+  kp.peers = static_cast<const __nv_bfloat16*>(peer_partials);
+  kp.send = static_cast<__nv_bfloat16*>(send_bufs);
   kp.prefetch = p->prefetch;
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out_shard);
@@ -2647,8 +2907,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   }
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
-  bool ok = make_map(&maps.a, A, g.M, g.K, kBK, kBM, true) &&
-            make_map(&maps.b, B, g.N, g.K, kBK, pair ? 128 : g.BN, true) &&
+  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d) &&
             make_map(&maps.c_st, base, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {

@@ -149,6 +149,10 @@ void build_tables(const Geometry& g, int order, int r, int x, int n_gemm_ctas, i
 }
 
 int finalize_plan(Plan* p) {
+  // The device copies of the tables (made by the first call that needs the device, which may be
+  // entwine_read_partial or a launch that failed later on) describe the plan as it was: drop them,
+  // the next call uploads the rebuilt tables.
+  if (p->dev) device_release(p);
   if (!p->num_sms_overridden) {
     int sms = device_sm_count();
     p->num_sms = sms > 0 ? sms : 148;
@@ -275,6 +279,20 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
     case ENTWINE_OPT_STAGES:
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);
+      return ENTWINE_OK;
+    case ENTWINE_OPT_REG_CONSUMER:
+      if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
+      p->reg_consumer = int(value);
+      return ENTWINE_OK;
+    case ENTWINE_OPT_KBLOCKS_PER_STAGE:
+      if (value < 0 || value > 2) return ENTWINE_ERR_INVALID;
+      p->kpb = int(value);
+      return ENTWINE_OK;
+    case ENTWINE_OPT_LDA:
+    case ENTWINE_OPT_LDB:
+      // rows start on 16-byte boundaries and do not overlap
+      if (value != 0 && (value < p->g.K || value % 8 != 0 || value > (int64_t(1) << 36))) return ENTWINE_ERR_INVALID;
+      (key == ENTWINE_OPT_LDA ? p->lda : p->ldb) = value;
       return ENTWINE_OK;
     case ENTWINE_OPT_PREFETCH:
       if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;

@@ -28,8 +28,9 @@ def _rows_to_f64(t, rows):
     return O.bf16_bits_to_f64(I.bits(t[rows]))
 
 
-@pytest.mark.parametrize("wl,r,orders,budgets", FULL, ids=lambda v: getattr(v, "name", None))
-def test_full_size_sampled_parity(wl, r, orders, budgets):
+def _sampled_parity(wl, r, orders, budgets):
+    """Sampled rows against the float64 oracle, every element against the properties that hold at
+    any size, exact counts; for each tile order and communication budget."""
     A, Bm = I.make_operands(wl, device="cuda")
     P = I.make_peer_partials(wl, device="cuda")
     R, W = wl.R, wl.W
@@ -81,34 +82,32 @@ def test_full_size_sampled_parity(wl, r, orders, budgets):
             assert not torch.isnan(out.float()).any()
             del Cd, acc, out, send
             p.destroy()
+    del A, Bm, P
+    torch.cuda.empty_cache()
 
 
-def test_sweep_corner_shapes_smoke_parity():
-    """Two corners of the sweep grid (smallest and a large one), both orders, budget 0 and 32:
-    exact counts and the any-size properties."""
-    for wl in (I.sweep_workloads()[0], I.sweep_workloads()[-4]):
-        A, Bm = I.make_operands(wl, device="cuda")
-        P = I.make_peer_partials(wl, device="cuda")
-        R, W, r = wl.R, wl.W, wl.W - 1
-        for order, n_comm in ((0, 0), (1, 32)):
-            p = E.Plan(wl.M, wl.N, wl.K, W, order, n_comm, rank=r)
-            out = torch.empty((R, wl.N), dtype=torch.bfloat16, device="cuda")
-            send = torch.empty((W - 1, R, wl.N), dtype=torch.bfloat16, device="cuda")
-            p.gemm_rs(A, Bm, P, out, send)
-            st = p.last_status()
-            c = p.counts()
-            assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
-            Cd = torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device="cuda")
-            p.read_partial(Cd)
-            ref = torch.matmul(A, Bm.t())          # library GEMM as a whole-matrix sanity check
-            assert (Cd.float() - ref.float()).abs().max() <= 0.02 * ref.float().abs().max()
-            for slot, d in enumerate(dd for dd in range(W) if dd != r):
-                assert torch.equal(send[slot], Cd[d * R:(d + 1) * R])
-            acc = Cd[r * R:(r + 1) * R].float()
-            for q in range(W - 1):
-                acc = acc + P[q, r * R:(r + 1) * R].float()
-            assert torch.equal(out, acc.to(torch.bfloat16))
-            p.destroy()
+@pytest.mark.parametrize("wl,r,orders,budgets", FULL, ids=lambda v: getattr(v, "name", None))
+def test_full_size_sampled_parity(wl, r, orders, budgets):
+    _sampled_parity(wl, r, orders, budgets)
+
+
+def _sweep_shape(M, K, W):
+    return next(w for w in I.sweep_workloads() if (w.M, w.K, w.W) == (M, K, W))
+
+
+# the four corners of the sweep grid (M x K_local, with the rank counts at the ends) and two
+# interior points; budgets at both ends and the middle of the sweep's range, both tile orders
+SWEEP_SAMPLE = [(2048, 512, 2), (32768, 4096, 8), (32768, 512, 2), (2048, 4096, 8), (8192, 1024, 4),
+                (16384, 2048, 8)]
+
+
+@pytest.mark.parametrize("M,K,W", SWEEP_SAMPLE)
+def test_sweep_shapes_sampled_parity(M, K, W):
+    """The sweep configuration against the oracle: sampled rows in float64, every element against
+    the any-size properties, exact counts."""
+    wl = _sweep_shape(M, K, W)
+    assert wl.K >= 256  # the float64 bound is feasible for a bf16-stored partial (see test_gpu_parity)
+    _sampled_parity(wl, W - 1 if M > 2048 else 0, (1, 0), (0, 16, 32))
 
 
 def test_ring_handover_keeps_every_element_exact():

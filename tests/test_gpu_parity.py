@@ -78,9 +78,9 @@ def _small(name, W, M, N, K, cid=9, idx=0):
 
 # sizes that span several tiles / blocks per CTA and ragged K (not a multiple of 64)
 SMALL = [
-    _small("s0", 2, 256, 256, 64, idx=0),
+    _small("s0_K64_vs_staged_model", 2, 256, 256, 64, idx=0),
     _small("s1", 2, 512, 512, 272, idx=1),     # K tail: 272 = 4*64 + 16
-    _small("s2", 4, 1024, 768, 80, idx=2),     # K tail: 80 = 64 + 16
+    _small("s2_K80_vs_staged_model", 4, 1024, 768, 80, idx=2),     # K tail: 80 = 64 + 16
     _small("s3", 3, 768, 384, 320, idx=3),     # BN = 128 only
     _small("s4", 8, 2048, 1024, 448, idx=4),
 ]
@@ -329,6 +329,10 @@ OPTION_SETS = [
     # release granularity (Sec. 5 ablation): groups of blocks, a partition, the whole output
     dict(release_group=3), dict(release_group=16), dict(release_group=-1), dict(release_group=-2),
     dict(release_group=5, pair_ctas=0), dict(release_group=-1, colocate=0, tail_help=0),
+    # how a stage of the operand ring is filled, and how the co-located consumer moves its tiles
+    dict(kblocks_per_stage=1), dict(kblocks_per_stage=2, stages=2), dict(kblocks_per_stage=1, stages=6),
+    dict(reg_consumer=0), dict(reg_consumer=0, kblocks_per_stage=2, stages=2), dict(reg_consumer=0, kblocks_per_stage=1),
+    dict(reg_consumer=0, pair_ctas=0), dict(reg_consumer=1, pair_ctas=0, kblocks_per_stage=1),
 ]
 
 
@@ -379,3 +383,82 @@ def test_many_ranks_small_steps():
         assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
         _check_against_oracle(wl, r, res, out, send)
         p.destroy()
+
+
+def test_every_configuration_is_checked_against_the_float64_bound():
+    """The staged-model branch above exists for the ragged-K test shapes (K = 64, 80) alone: the
+    five configurations the tolerance is stated for, and every sweep shape, take the float64
+    oracle."""
+    for wl in list(I.CONFIGS.values()) + I.sweep_workloads():
+        assert _tolerance_is_feasible(wl), wl.name
+
+
+def test_pre_launch_options_after_the_device_tables_exist():
+    """entwine_read_partial (or a launch that failed late) creates the plan's device tables before
+    the first launch; an option that rebuilds the host tables afterwards must reach the device
+    too: more lists than before, another rank, another block width, then a checked launch."""
+    wl = SMALL[4]
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    p = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=0)
+    Cd = torch.empty((wl.M, wl.N), dtype=torch.bfloat16, device="cuda")
+    p.read_partial(Cd)              # device tables of the 4-list, rank-0 plan now exist
+    torch.cuda.synchronize()
+    p.set_option(E.OPT_LISTS, 37)   # many more lists than the first tables had
+    p.set_option(E.OPT_RANK, 5)
+    p.set_option(E.OPT_BLOCK_N, 128)
+    c = p.counts()
+    assert c["x"] == 37
+    res = O.gemm_rs(Ab, Bb, Pb, 5, wl.W, 128, 1, 37)
+    assert (p.export(E.EXPORT_TASKS).reshape(-1, 8) == res["maps"][0]).all()
+    out, send = _alloc_outputs(wl)
+    p.gemm_rs(A.cuda(), Bm.cuda(), P.cuda(), out, send)
+    st = p.last_status()
+    assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+    _check_against_oracle(wl, 5, res, out, send)
+    # after a launch the same options are refused
+    with pytest.raises(E.EntwineError):
+        p.set_option(E.OPT_LISTS, 8)
+    p.destroy()
+
+
+@pytest.mark.parametrize("wl", [SMALL[1], SMALL[4]], ids=lambda w: w.name)
+def test_leading_dimensions(wl):
+    """A and B as row-padded views (ENTWINE_OPT_LDA / LDB): same bits as the contiguous call, for
+    one and two k-blocks per stage, CTA pairs and single CTAs, and a ragged K."""
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    Ad, Bd, Pd = A.cuda(), Bm.cuda(), P.cuda()
+    lda, ldb = wl.K + 8, wl.K + 72
+    Apad = torch.full((wl.M, lda), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Bpad = torch.full((wl.N, ldb), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Apad[:, :wl.K] = Ad
+    Bpad[:, :wl.K] = Bd
+    r = 1
+    res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, 1, 4)
+    for opts in (dict(), dict(kblocks_per_stage=1), dict(pair_ctas=0)):
+        p0 = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, **opts)
+        out0, send0 = _alloc_outputs(wl)
+        p0.gemm_rs(Ad, Bd, Pd, out0, send0)
+        p0.last_status()
+        p0.destroy()
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, lda=lda, ldb=ldb, **opts)
+        out, send = _alloc_outputs(wl)
+        p.gemm_rs(Apad, Bpad, Pd, out, send)
+        p.last_status()
+        _check_against_oracle(wl, r, res, out, send)
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        # back to contiguous operands on the same plan
+        p.set_option(E.OPT_LDA, 0)
+        p.set_option(E.OPT_LDB, 0)
+        out.fill_(float("nan"))
+        p.gemm_rs(Ad, Bd, Pd, out, send)
+        p.last_status()
+        assert torch.equal(out, out0)
+        p.destroy()
+    with pytest.raises(E.EntwineError):
+        E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 4, lda=wl.K + 4)      # not a multiple of 8 elements
+    with pytest.raises(E.EntwineError):
+        E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 4, ldb=wl.K - 8)      # rows would overlap

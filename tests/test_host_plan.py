@@ -130,6 +130,14 @@ def test_fig3_example_through_the_library(golden):
         red = [int(t[2]) for t in tasks if t[0] == 0 and t[4] == j]
         assert red == [int(v) for v in g[key][0]]
     p.destroy()
+    # the push lists of both traversals, as the library's planner builds them
+    for name, order in (("push_interleaved", E.ORDER_INTERLEAVED), ("push_grouped", E.ORDER_ROW_MAJOR)):
+        p = E.Plan(M, N, 64, W, order, x, num_sms=148, block_n=BN, rank=r)
+        tasks = p.export(E.EXPORT_TASKS).reshape(-1, 8)
+        for j in range(2):
+            want = [tuple(int(v) for v in e.split(":")) for e in g[f"{name}_C{j}"][0]]
+            assert [(int(t[1]), int(t[2])) for t in tasks if t[0] == 1 and t[4] == j] == want
+        p.destroy()
 
 
 def test_launch_without_device_fails_loudly():

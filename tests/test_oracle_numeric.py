@@ -225,8 +225,12 @@ def test_layer_chain_is_residual_add_then_rmsnorm():
     assert np.allclose((n1 ** 2).mean(-1), 1.0, rtol=1e-12)
 
 
-def test_norm_task_order_covers_every_tile_band_by_band():
-    order = O.norm_task_order(1024, 768, 4)
-    rowsT, nTn = 1024 // 4 // 128, 768 // 128
-    assert order.shape == (rowsT * nTn, 2)
-    assert [tuple(v) for v in order] == [(b, c) for b in range(rowsT) for c in range(nTn)]
+def test_norm_task_order_hand_listed():
+    """Two bands of three tile columns (R = 256 rows per rank, N = 384), listed by hand: band 0's
+    tiles left to right, then band 1's.  A column-first walk, a band-last walk or a transposed
+    (column, band) pair would each differ from this list."""
+    order = O.norm_task_order(512, 384, 2)
+    assert order.dtype == np.int32
+    assert order.tolist() == [[0, 0], [0, 1], [0, 2], [1, 0], [1, 1], [1, 2]]
+    # one band only: W = 4 leaves R = 128
+    assert O.norm_task_order(512, 384, 4).tolist() == [[0, 0], [0, 1], [0, 2]]

@@ -39,6 +39,13 @@ def test_fig3_worked_example(golden):
     for j in range(2):
         assert [t for (kind, d, t, k) in lists2[j] if kind == O.KIND_REDUCE] == \
                [t for (kind, d, t, k) in lists[j] if kind == O.KIND_REDUCE]
+    # the push lists do: non-owned tiles are dealt out in the order their flags are published
+    # (hand-written vectors for both traversals; numbering by (d, t) instead would fail the
+    # interleaved one, numbering by position alone would fail the split between C0 and C1)
+    for name, ls in (("push_interleaved", lists), ("push_grouped", lists2)):
+        for j in range(2):
+            want = [tuple(int(v) for v in e.split(":")) for e in g[f"{name}_C{j}"][0]]
+            assert [(d, t) for (kind, d, t, k) in ls[j] if kind == O.KIND_PUSH] == want
 
 
 def _longest_local_run(dest, r):
@@ -255,9 +262,3 @@ def test_geometry_rejects_bad_shapes():
                 (256, 384, 2, 256), (256, 256, 2, 64)]:
         with pytest.raises(ValueError):
             O.Geometry(*bad)
-
-
-def test_completion_log_validator():
-    assert O.valid_completion_log([0, 2, 1, 3], 4, 2)
-    assert not O.valid_completion_log([2, 0, 1, 3], 4, 2)      # CTA 0 ran 2 before 0
-    assert not O.valid_completion_log([0, 1, 1, 3], 4, 2)      # not a permutation
