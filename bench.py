@@ -30,9 +30,14 @@ sys.path.insert(0, ROOT)
 METRIC = "fused GEMM-RS TFLOP/s and fraction of max(tensor peak, HBM) roofline"
 # Peaks measured on this machine (used only if MEASURED_PEAKS.json is absent).
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic (bytes read + written per launch) of the fused kernel from an ncu capture of
-# the named workload; see profiles/.  None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"attn_out_proj": 53.69e6, "mlp_down_proj": 845.38e6, "short_k_comm_bound": 507.35e6}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of the fused kernel from
+# the ncu capture of the named workload that profiles/ summarises; the summary file is carried
+# beside the number so that a stale figure can be told from a fresh one.
+NCU_TRAFFIC = {
+    "attn_out_proj": {"bytes": 53.69e6, "summary": "profiles/fused_kernel_attn_out_proj.md"},
+    "mlp_down_proj": {"bytes": 845.38e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+    "short_k_comm_bound": {"bytes": 507.35e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+}
 # Launch configuration per workload: communication SMs, tile order.
 # Launch configuration per workload (the best point of a budget x order scan on B200): number of
 # dedicated communication SMs (0 = consumer warps co-located with the producer in every CTA),
@@ -166,13 +171,28 @@ def _dist_env():
         int(os.environ.get("WORLD_SIZE", "1"))
 
 
+def blas_threads():
+    """Threads of the BLAS pool behind numpy's matmul (what the oracle's float64 GEMM runs on),
+    after setting it to the cores this process may use."""
+    cores = len(os.sched_getaffinity(0))
+    try:
+        import threadpoolctl
+        threadpoolctl.threadpool_limits(limits=cores, user_api="blas")
+        pools = [p for p in threadpoolctl.threadpool_info() if p.get("user_api") == "blas"]
+        if pools:
+            return max(int(p["num_threads"]) for p in pools)
+    except Exception:
+        pass
+    return cores
+
+
 def run_cpu_oracle(wl, launch, rows_per_pass, passes):
     """Times the oracle (float64 GEMM of the sampled rows + reduce-scatter definition + the
-    whole integer schedule) and returns (best seconds, flops of one pass, threads used)."""
+    whole integer schedule) and returns (seconds per pass, flops of one pass, threads used)."""
     import numpy as np
-    import torch
     from oracle import entwine_oracle as O
     from paper_2609_11562_b200 import inputs as I
+    threads = blas_threads()
     A, Bm = I.make_operands(wl)
     P = I.make_peer_partials(wl)
     Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
@@ -186,7 +206,7 @@ def run_cpu_oracle(wl, launch, rows_per_pass, passes):
         O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, launch["order"], x, rows=rows)
         times.append(time.perf_counter() - t0)
     n_rows = wl.M if full else rows_per_pass
-    return times, 2.0 * n_rows * wl.N * wl.K, torch.get_num_threads()
+    return times, 2.0 * n_rows * wl.N * wl.K, threads
 
 
 def main_reference(args, wl, launch):
@@ -253,6 +273,7 @@ def measure_workload(wl, launch, steps, warmup, flush, torch, E, I, detailed):
     st = plan.last_status()
     res["fused_us"] = us
     res["status"] = st
+    res["sm_mhz"] = plan.last_sm_clock_mhz()
     res["fused_hot_us"] = time_steps(lambda: plan.gemm_rs(A, Bm, P, out, send), steps, 3, flush, torch, cold=False)
     plan.last_status()
     # Back to back: `steps` calls queued between ONE event pair, no flush.  The queue hides the
@@ -363,6 +384,20 @@ def run_sweep(args, peaks, flush, torch, E, I):
                     st = plan.last_status()
                     c = plan.counts()
                     assert st["tiles_reduced"] == c["n_reduce"] and st["tiles_pushed"] == c["n_push"]
+                    if n_comm == I.SWEEP_COMM_SMS[0]:
+                        # the properties that hold at any size, once per shape and order: what was
+                        # pushed is the stored partial, what was reduced is its fp32 rank-order sum
+                        r, R = wl.W - 1, wl.R
+                        Cd = torch.empty(wl.M, wl.N, dtype=torch.bfloat16, device="cuda")
+                        plan.read_partial(Cd)
+                        torch.cuda.synchronize()
+                        for slot, d in enumerate(dd for dd in range(wl.W) if dd != r):
+                            assert torch.equal(send[slot], Cd[d * R:(d + 1) * R])
+                        acc = Cd[r * R:(r + 1) * R].float()
+                        for q in range(wl.W - 1):
+                            acc = acc + P[q, r * R:(r + 1) * R].float()
+                        assert torch.equal(out, acc.to(torch.bfloat16))
+                        del Cd, acc
                     med = statistics.median(us)
                     rec = {"M": wl.M, "N": wl.N, "K_local": wl.K, "W": wl.W, "n_comm_sms": n_comm,
                            "tile_order": "interleaved" if order else "row_major", "fused_us": med,
@@ -444,8 +479,8 @@ def run_ablation(args, peaks, flush, torch, E, I):
         report[wl.name] = rec
         del A, Bm, P, out, send
         torch.cuda.empty_cache()
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "ablation.json"), "w") as f:
+    os.makedirs(args.out_dir, exist_ok=True)
+    with open(os.path.join(args.out_dir, "ablation.json"), "w") as f:
         json.dump(report, f, indent=1)
     print(json.dumps({"ablation": report}))
     return 0
@@ -511,8 +546,8 @@ def run_layer_chain(args, peaks, flush, torch, E, I):
         }
         del A, Bm, P, res, w, hidden, normed, out, send, Cfull
         torch.cuda.empty_cache()
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "layer_chain.json"), "w") as f:
+    os.makedirs(args.out_dir, exist_ok=True)
+    with open(os.path.join(args.out_dir, "layer_chain.json"), "w") as f:
         json.dump(report, f, indent=1)
     print(json.dumps({"layer_chain": report}))
     return 0
@@ -523,18 +558,21 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="attn_out_proj")
+    ap.add_argument("--workload", default="mlp_down_proj",
+                    help="default: the largest single-GPU configuration (MLP down-projection)")
+    ap.add_argument("--out-dir", default=os.path.join(ROOT, "bench_out"),
+                    help="where --sweep, --ablation and --layer-chain write their JSON files")
     ap.add_argument("--impl", default="entwine", choices=["entwine", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations and comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="run the sweep configuration (60 shapes x budgets 0..32 x both orders), write one "
                          "JSON line per point to --sweep-out and print a summary line")
-    ap.add_argument("--sweep-out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
+    ap.add_argument("--sweep-out", default=None, help="default: <out-dir>/sweep.jsonl")
     ap.add_argument("--sweep-iters", type=int, default=8)
     ap.add_argument("--ablation", action="store_true",
                     help="the design ablations (computation order, release granularity, SM sharing) on a "
-                         "short-K and a long-K shape; prints one JSON line and writes gpurun_out/ablation.json")
+                         "short-K and a long-K shape; prints one JSON line and writes <out-dir>/ablation.json")
     ap.add_argument("--layer-chain", action="store_true",
                     help="GEMM-RS + residual add + RMSNorm in one launch against library kernels for the rest "
                          "(attention output of a 70B-shaped layer, three sequence lengths)")
@@ -546,6 +584,8 @@ def main():
                     help="profiling aid: run warmup+steps launches of one mode on the workload and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "entwine" else args.warmup
+    if args.sweep_out is None:
+        args.sweep_out = os.path.join(args.out_dir, "sweep.jsonl")
 
     from paper_2609_11562_b200 import inputs as I
     apply_tuned_table()
@@ -661,6 +701,7 @@ def main():
                          "timed region shorter than the sampling period: same load continued untimed")
     us = [a.elapsed_time(b) * 1e3 for a, b in evs]
     status = plan.last_status()
+    kernel_mhz = plan.last_sm_clock_mhz()  # cycle counter against the global timer inside the last timed launch
     total_us = max_over_ranks(sum(us), dist, "cuda")
     mean_us = total_us / args.steps
     value = whole_job_tflops(world, wl.flops, mean_us * 1e-6)
@@ -728,7 +769,8 @@ def main():
     # cap, and the nominal HBM bandwidth
     t_alt = max(wl.flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12), wl.comm_bytes / 8.0e12)
     roof["frac_vs_sustained_tensor_and_nominal_hbm"] = t_alt / (mean_us * 1e-6)
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
+    roof["traffic"] = NCU_TRAFFIC.get(wl.name, {}).get("bytes")
+    roof["traffic_source"] = NCU_TRAFFIC.get(wl.name, {}).get("summary")
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
     roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
     roof["kernel"] = "entwine_fused_kernel<256, true, false, false>"
@@ -744,7 +786,8 @@ def main():
                    "block": "128x256 blocks on CTA pairs (256x256 pair tiles)",
                    "emulated_rank": launch["rank"], "l2": "flushed between timed steps (512 MiB memset)",
                    "multi_gpu": "replicas only"},
-        "us_per_call": {"mean": mean_us, "median": statistics.median(us), "min": min(us)},
+        "us_per_call": {"mean": mean_us, "median": statistics.median(us), "min": min(us),
+                        "sm_mhz_inside_kernel": kernel_mhz, "mean_us_times_sm_mhz": mean_us * kernel_mhz},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roof,
         "device_status": {"t_gemm_us": status["t_gemm_ns"] / 1e3, "t_end_us": status["t_end_ns"] / 1e3,
                           "tail_us": (status["t_end_ns"] - status["t_gemm_ns"]) / 1e3},
@@ -768,6 +811,8 @@ def main():
                 "fused_back_to_back_us": r["fused_back_to_back_us"],
                 "fused_graph_replay_us": r["fused_graph_replay_us"],
                 "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
+                "roofline_frac_back_to_back": max(tc, hb) * 1e6 / r["fused_back_to_back_us"],
+                "sm_mhz_inside_kernel": r["sm_mhz"], "fused_us_times_sm_mhz": fused * r["sm_mhz"],
                 "bound": "tensor" if tc >= hb else "hbm",
                 "unfused_cublas_then_reduce_us": med(r["unfused_us"]),
                 "speedup_vs_unfused": med(r["unfused_us"]) / fused,

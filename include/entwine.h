@@ -292,6 +292,15 @@ int entwine_plan_export(entwine_plan_t plan, int what, void* host_buf, size_t* b
 int entwine_last_status(entwine_plan_t plan, int64_t out[8]);
 
 /*
+ * entwine_last_sm_clock - how fast the SMs really ran during the launch that the last
+ * entwine_last_status call reported: out[0] = SM cycles and out[1] = nanoseconds that CTA 0
+ * spent in the kernel (cycle counter against the global timer).  cycles / ns = GHz.  Times
+ * measured on a power-limited part are read against this clock, not the nominal one.  Host
+ * only (no synchronisation); zeros before the first status read.
+ */
+int entwine_last_sm_clock(entwine_plan_t plan, int64_t out[2]);
+
+/*
  * entwine_gemm_rs_static - entwine_gemm_rs for callers that must not allocate.  (The paper
  * has no counterpart; this entry point exists for the library's users only.)
  *

@@ -53,7 +53,7 @@ struct StatusSlot {
   unsigned long long t_start;     // min globaltimer at CTA entry
   unsigned long long t_gemm_end;  // max globaltimer after a producer CTA's last block
   unsigned long long t_end;       // max globaltimer at CTA exit
-  unsigned long long pad;
+  unsigned long long clock;       // CTA 0: SM cycles << 32 | ns between its start and its exit
 };
 static_assert(sizeof(StatusSlot) == 64, "StatusSlot layout");
 

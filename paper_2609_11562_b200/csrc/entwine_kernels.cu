@@ -13,6 +13,36 @@
 
 #include "entwine_internal.h"
 
+// Optional per-role wait-time counters (builds with -DENTWINE_PROFILE only; off in the product):
+// cycles a role spent waiting at each of its synchronisation points, per CTA.
+#ifdef ENTWINE_PROFILE
+__device__ unsigned long long g_prof[256 * 16];
+extern "C" int entwine_debug_read_profile(void* dst, int clear) {
+  cudaError_t e = cudaMemcpyFromSymbol(dst, g_prof, sizeof(g_prof));
+  if (e == cudaSuccess && clear) {
+    static unsigned long long zeros[256 * 16];
+    e = cudaMemcpyToSymbol(g_prof, zeros, sizeof(zeros));
+  }
+  return (int)e;
+}
+// a role accumulates in a register array and writes it out once, at its end
+#define PROF_DECL() unsigned long long prof_acc_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define PROF_T0() const long long prof_t0_ = clock64()
+#define PROF_ADD(k) (prof_acc_[k] += (unsigned long long)(clock64() - prof_t0_))
+#define PROF_FLUSH(cond)                                                        \
+  do {                                                                          \
+    if (cond) {                                                                 \
+      for (int k_ = 0; k_ < 16; ++k_)                                           \
+        if (prof_acc_[k_]) atomicAdd(&g_prof[blockIdx.x * 16 + k_], prof_acc_[k_]); \
+    }                                                                           \
+  } while (0)
+#else
+#define PROF_DECL() do { } while (0)
+#define PROF_T0() do { } while (0)
+#define PROF_ADD(k) do { } while (0)
+#define PROF_FLUSH(cond) do { } while (0)
+#endif
+
 namespace entwine {
 
 // ------------------------------------------------------------------------------------------
@@ -34,23 +64,23 @@ constexpr int kEpiWarp0 = 4;      // producer: epilogue warps 4..7
 constexpr int kEpiThreads = 128;
 constexpr int kRedWarp0 = 8;      // consumer: reducing warps 8..15
 constexpr int kRedThreads = 256;
-constexpr int kCStoreWarp = 16;   // producer: TMA stores of the partial C
+constexpr int kSpareWarp = 16;    // (no role: keeps the flag warp on the sub-core it was measured on)
 constexpr int kFlagWarp = 17;     // producer: releases the tile flags of stored blocks
 constexpr int kGemmThreads = 256; // warps 0, 1, 4-7, 16, 17
 constexpr uint32_t kSpinCheck = 128;  // spins between looks at the timer / abort flag
-constexpr int kEpiBufBytes = 16384;   // one staging buffer: 128 rows x 64 columns of bf16, 128B-swizzled
+constexpr int kEpiWarpBytes = 4096;   // an epilogue warp's staging: its 32 rows x 64 columns of bf16, 128B-swizzled
 
 // Shared-memory map (offsets from a 1024-byte aligned base).  The first 224 KiB are split at
 // launch time between the producer's operand ring (S stages), the epilogue staging and the
 // consumer's ring A, which a producer CTA's consumer warps use while it still produces:
 //   [0, S*stage)                operand ring of the producer
-//   [S*stage, S*stage + 32 KiB) epilogue staging (2 x 16 KiB)
+//   [S*stage, S*stage + 16 KiB) epilogue staging (4 KiB per epilogue warp)
 //   [.., 229376)                consumer ring A (32 KiB with 5 pair stages, 64 KiB with 4, ...)
 //   [0, 196608)                 consumer ring B: 6 slots of 32 KiB, used once the CTA's producer
 //                               work is over (and by dedicated consumer CTAs from the start)
 //   [229376, 230016)            mbarriers, TMEM base slot
 constexpr int kDataBytes = 229376;
-constexpr int kStagingBytes = 2 * kEpiBufBytes;
+constexpr int kStagingBytes = 4 * kEpiWarpBytes;
 constexpr int kRingBOff = 0;
 constexpr int kRingBBytes = 196608;
 constexpr int kMaxSlots = 8;
@@ -120,6 +150,7 @@ struct KParams {
   // memory
   __nv_bfloat16* out;            // out_shard [R][N] (written by the reducing warps)
   const __nv_bfloat16* cws;      // the rank's partial C [M][N] as the consumer reads it (register path)
+  __nv_bfloat16* cws_out;        // ... as the producer's epilogue writes it
   const __nv_bfloat16* peers;    // incoming partials [W-1][M][N] (register path; pull mode: see heap)
   __nv_bfloat16* send;           // send_bufs [W-1][R][N] (register path)
   long long heap_buf_off;        // pull mode: offset of this call's partial-output buffer inside a segment
@@ -395,6 +426,9 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
 __device__ __forceinline__ void st_release_cta(int* p, int v) {
   asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_release_cta_add(int* p, int v) {
+  asm volatile("red.release.cta.shared::cta.add.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
 __device__ __forceinline__ int ld_acquire_cta(const int* p) {
   int v;
   asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
@@ -512,7 +546,7 @@ struct CtaShared {
   volatile int stages_free;  // the CTA's last MMA has completed: its operand stages are free
   int ring_b_bytes;          // size of this CTA's ring B: the operand stages of a producer CTA (ring B
                              // then starts before the epilogue is over), 192 KiB of a consumer CTA
-  int blocks_stored;       // blocks of this CTA whose partial-C stores are complete
+  int warps_stored;        // epilogue warps x blocks of this CTA whose partial-C stores have been issued
   float inv_rms[kTile];    // layer chain: 1 / RMS of the rows of the tile being normalised
   SlotMeta meta[2][kMaxSlots];
 };
@@ -729,6 +763,7 @@ template <bool NORM, bool PULL>
 __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, uint32_t smem_base, Ring ring) {
   const int lane = threadIdx.x & 31;
   const int ctid = threadIdx.x - kRedWarp0 * 32;
+  PROF_DECL();
   int slot = -1;
   uint32_t ph = 0;
   // layer chain: this thread's 8 chunks (16 bytes each) of the residual of the tile being
@@ -741,7 +776,11 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
     if (++slot == ring.n_slots) { slot = 0; ph ^= 1; }
     // one lane per warp polls; the warp-level vote carries the barrier's acquire to all lanes
     bool landed = true;
-    if (lane == 0) landed = mbar_wait(ring.full(slot), ph, P, sh);
+    if (lane == 0) {
+      PROF_T0();
+      landed = mbar_wait(ring.full(slot), ph, P, sh);
+      if (ctid == 0) PROF_ADD(12);
+    }
     if (!__all_sync(0xffffffffu, landed)) {
       sh->abort = 1;
       break;
@@ -756,12 +795,16 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
     }
     if (!NORM && m.kind == 4) {
       // a whole reduce task from registers (ReduceTile of Sec. 4.2 on all 128 rows of the tile)
+      PROF_T0();
       if (P.W == 2) reg_reduce_tile<2, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       else if (P.W == 4) reg_reduce_tile<4, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       else if (P.W == 8) reg_reduce_tile<8, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       else reg_reduce_tile_any<PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
+      if (ctid == 0) PROF_ADD(10);
     } else if (!NORM && !PULL && m.kind == 5) {
+      PROF_T0();
       reg_push_tile(P, ctid, m.dst_x, m.aux, m.dst_y);
+      if (ctid == 0) PROF_ADD(11);
     } else if (!NORM && m.kind == 0) {
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
       const int rs = ring.rs, sub_bytes = ring.sub_bytes;
@@ -879,6 +922,7 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
     __syncwarp();
     if (lane == 0) mbar_arrive(ring.red(slot));
   }
+  PROF_FLUSH(ctid == 0);
 }
 
 // One CTA's consumer work, run by warps 2, 3 and 8-15.  Warp 2 claims tasks from `n_lists`
@@ -896,6 +940,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
 
   if (warp == kCommWarp) {
     // ---------------- claim, poll, load ----------------
+    PROF_DECL();
     // tiles are read once: ask L2 to evict them first so that the producer's operand panels stay
     const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     int it = 0;
@@ -1113,12 +1158,14 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             const int own = __shfl_sync(0xffffffffu, k_own, src);
             const int t = __shfl_sync(0xffffffffu, k_t, src);
             bool mine_ok = true;
+            PROF_T0();
             if (lane == 0) mine_ok = wait_flag<false>(&P.flags_own[own], P);
             else if (kind == 0) {
               for (int q = lane - 1; mine_ok && q < P.W - 1; q += 31)
                 mine_ok = wait_flag<PULL>(&P.flags_peer[peer_row(q) * P.Q + t], P);
             }
             ok = __all_sync(0xffffffffu, mine_ok);
+            if (lane == 0) PROF_ADD(13);
             if (!ok) {
               if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, base + i);
               break;
@@ -1132,7 +1179,11 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             bool slot_ok = true;
             if (lane == 0) {
               const int slot = it % ring.n_slots;
-              slot_ok = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+              {
+                PROF_T0();
+                slot_ok = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+                PROF_ADD(14);
+              }
               if (slot_ok) {
                 SlotMeta& m = sh->meta[0][slot];
                 m.kind = 4 + kind;
@@ -1279,6 +1330,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         issue_norm_run(i, kRun);
       }
     }
+    PROF_FLUSH(lane == 0);
     // end-of-work marker so that the other consumer warps leave their loops
     if (lane == 0) {
       const int slot = it % ring.n_slots;
@@ -1393,6 +1445,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ CtaShared sh;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  PROF_DECL();
   StatusSlot* st = &P.status[P.seq & 1];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t smem_base = smem_u32(smem);
@@ -1433,10 +1486,19 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     nx->t_start = ~0ULL;
     nx->t_gemm_end = 0;
     nx->t_end = 0;
+    nx->clock = 0;
+  }
+  // CTA 0 times itself with the SM's cycle counter and the global timer: their ratio is the SM
+  // clock this launch really ran at
+  long long clk0 = 0;
+  unsigned long long ns0 = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    clk0 = clock64();
+    ns0 = globaltimer_ns();
   }
   if (threadIdx.x == 0) {
     sh.abort = 0;
-    sh.blocks_stored = 0;
+    sh.warps_stored = 0;
     sh.gemm_done = (is_producer && n_my > 0) ? 0 : 1;
     sh.stages_free = (is_producer && n_my > 0) ? 0 : 1;
     sh.ring_b_bytes = (is_producer && n_my > 0 && P.early_b) ? P.stage_area : kRingBBytes;
@@ -1477,7 +1539,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
 
   CommCounters cnt;
   unsigned published = 0;
-  const bool gemm_warp = warp == kTmaWarp || warp == kMmaWarp || warp == kCStoreWarp || warp == kFlagWarp ||
+  const bool gemm_warp = warp == kTmaWarp || warp == kMmaWarp || warp == kSpareWarp || warp == kFlagWarp ||
                          (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4);
   const bool comm_warp = warp == kCommWarp || warp == kStoreWarp ||
                          (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32);
@@ -1508,7 +1570,12 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
         const int b_row = nb * BN + (PAIR ? (int)cta_rank * C::kBRows : 0);
         for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1, P, &sh)) { ok = false; break; }
+          {
+            PROF_T0();
+            const bool got = mbar_wait(empty_bar(stage), phase ^ 1, P, &sh);
+            PROF_ADD(0);
+            if (!got) { ok = false; break; }
+          }
           const uint32_t a_dst = smem_base + stage * stage_bytes;
           const uint32_t b_dst = a_dst + P.kpb * C::kABytes;
           // k-blocks of this stage that exist (a ragged last stage is filled, and multiplied, in part)
@@ -1555,12 +1622,25 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       uint32_t acc_phase = 0;
       constexpr uint32_t idesc = instr_desc<BN, PAIR ? 256 : 128>();
       bool ok = true;
+#ifdef ENTWINE_PROFILE
+      const long long prof_mma0 = clock64();
+#endif
       for (int i = 0; ok && i < n_my; ++i) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh)) { ok = false; break; }
+        {
+          PROF_T0();
+          const bool got = mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh);
+          PROF_ADD(1);
+          if (!got) { ok = false; break; }
+        }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
-          if (!mbar_wait(full_bar(stage), phase, P, &sh)) { ok = false; break; }
+          {
+            PROF_T0();
+            const bool got = mbar_wait(full_bar(stage), phase, P, &sh);
+            PROF_ADD(2);
+            if (!got) { ok = false; break; }
+          }
           tc_fence_after();
           const uint32_t a_s = smem_base + stage * stage_bytes;
           const uint32_t b_s = a_s + P.kpb * C::kABytes;
@@ -1585,19 +1665,36 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         else tc_commit(tfull_bar(acc));
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
+#ifdef ENTWINE_PROFILE
+      prof_acc_[8] += (unsigned long long)(clock64() - prof_mma0);
+#endif
       if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -2); }
     } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
-      // ---- epilogue: TMEM -> bf16 -> swizzled staging.  The block leaves as BN/64 boxes of
-      //      128 rows x 64 columns through two staging buffers; the publishing warp stores them,
-      //      so these warps never wait for global memory ----
+      // ---- epilogue: TMEM -> bf16 -> global.  A warp owns 32 rows of the block (its TMEM lane
+      //      quarter).  Its threads round their rows to bf16 into the warp's own swizzled staging
+      //      (32 rows x 128 bytes), the warp reads that back row-wise and stores whole 128-byte
+      //      lines of the partial C with plain 16-byte stores: no other warp, no copy engine and no
+      //      buffer hand-over lies between the accumulator and memory.  After a block's stores
+      //      the warp counts itself in warps_stored (release); the flag warp publishes the
+      //      block's tiles when all four have (Sec. 4.2: flags after all of the block's stores) ----
       const int q = warp & 3;  // TMEM lane quarter this warp may read = its 32 rows of the block
-      const uint32_t stg0 = smem_base + n_stages * stage_bytes + (q * 32 + lane) * 128;
+      const uint32_t wstage = smem_base + n_stages * stage_bytes + q * kEpiWarpBytes;
+      const uint32_t my_row = wstage + lane * 128;
       int acc = 0;
       uint32_t acc_phase = 0;
-      int nbox = 0;  // boxes staged so far: buffer nbox & 1, use (nbox >> 1)
       bool ok = true;
+#ifdef ENTWINE_PROFILE
+      const long long prof_epi0 = clock64();
+#endif
       for (int i = 0; ok && i < n_my; ++i) {
-        ok = mbar_wait(tfull_bar(acc), acc_phase, P, &sh);
+        int d, l;
+        block_of(i, &d, &l);
+        const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
+        {
+          PROF_T0();
+          ok = mbar_wait(tfull_bar(acc), acc_phase, P, &sh);
+          if (warp == kEpiWarp0 && lane == 0) PROF_ADD(3);
+        }
         ok = __all_sync(0xffffffffu, ok);  // reconverge; the warp leaves the loop together
         if (!ok) break;
         tc_fence_after();
@@ -1607,92 +1704,117 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           sh.stages_free = 1;
         }
         const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + acc * BN;
-#pragma unroll 1
-        for (int j = 0; j < BN / 64; ++j, ++nbox) {
-          const int buf = nbox & 1;
-          bool free_buf = true;
-          if (lane == 0) free_buf = mbar_wait(sfree_bar(buf), ((nbox >> 1) & 1) ^ 1, P, &sh);
-          ok = __all_sync(0xffffffffu, free_buf);
-          if (!ok) break;
-          const uint32_t row = stg0 + buf * kEpiBufBytes;
+        // this lane's share of a read-back: row (lane / 8) + 4 * it of the warp's 32, 16-byte chunk lane % 8
+        __nv_bfloat16* const cdst = P.cws_out + (long long)(mb * kBM + q * 32 + (lane >> 3)) * P.N + nb * BN + (lane & 7) * 8;
+        // Two register sets: the TMEM load of the next 32 columns is in flight while the previous
+        // 32 are rounded and staged (a tcgen05.ld takes a few hundred cycles).
+        uint32_t va[32], vb[32];
+        // rounds 32 fp32 values of this thread's row to bf16 (nearest even) and writes them as
+        // four 16-byte chunks of the row's 128 swizzled bytes
+        auto stage32 = [&](const uint32_t (&v)[32], int cc) {
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(taddr + j * 64 + cc * 32, v);
-            tmem_ld_wait();
-            if (j == BN / 64 - 1 && cc == 1) {
-              // last read of this accumulator: the MMA warp may overwrite it
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) {
-                if (leader) mbar_arrive(tempty_bar(acc));
-                else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
-              }
+          for (int e = 0; e < 4; ++e) {
+            uint4 o;
+            uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * e + 2 * u]),
+                                                        __uint_as_float(v[8 * e + 2 * u + 1]));
+              ow[u] = *reinterpret_cast<uint32_t*>(&hh);
             }
+            const int chunk = cc * 4 + e;  // 16-byte chunk inside the 128-byte row
+            st_shared_v4(my_row + ((chunk ^ (lane & 7)) << 4), o);
+          }
+        };
+#if defined(ENTWINE_EXP) && ENTWINE_EXP == 3
+        // each lane writes its own row: 64 bytes per 32 columns, as four 16-byte stores
+        __nv_bfloat16* const crow = P.cws_out + (long long)(mb * kBM + q * 32 + lane) * P.N + nb * BN;
+        auto direct32 = [&](const uint32_t (&v)[32], int col) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              uint4 o;
-              uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
+          for (int e = 0; e < 4; ++e) {
+            uint4 o;
+            uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * e + 2 * u]),
-                                                          __uint_as_float(v[8 * e + 2 * u + 1]));
-                ow[u] = *reinterpret_cast<uint32_t*>(&hh);
-              }
-              const int chunk = cc * 4 + e;  // 16-byte chunk inside the 128-byte row
-              st_shared_v4(row + ((chunk ^ (lane & 7)) << 4), o);
+            for (int u = 0; u < 4; ++u) {
+              __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * e + 2 * u]),
+                                                        __uint_as_float(v[8 * e + 2 * u + 1]));
+              ow[u] = *reinterpret_cast<uint32_t*>(&hh);
+            }
+            __stcg(reinterpret_cast<uint4*>(crow + col + e * 8), o);
+          }
+        };
+        tmem_ld32(taddr, va);
+#pragma unroll 1
+        for (int j = 0; j < BN / 64; ++j) {
+          tmem_ld_wait();
+          tmem_ld32(taddr + j * 64 + 32, vb);
+          direct32(va, j * 64);
+          tmem_ld_wait();
+          if (j + 1 < BN / 64) {
+            tmem_ld32(taddr + (j + 1) * 64, va);
+          } else {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (leader) mbar_arrive(tempty_bar(acc));
+              else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
             }
           }
-          fence_async_smem();  // the TMA store reads what this warp wrote
-          __syncwarp();
-          if (lane == 0) mbar_arrive(staged_bar(buf));
+          direct32(vb, j * 64 + 32);
         }
+#else
+        tmem_ld32(taddr, va);
+#pragma unroll 1
+        for (int j = 0; j < BN / 64; ++j) {
+          tmem_ld_wait();                                // columns [64 j, 64 j + 32) are in va
+          tmem_ld32(taddr + j * 64 + 32, vb);
+#if !defined(ENTWINE_EXP) || ENTWINE_EXP != 2
+          stage32(va, 0);
+#endif
+          tmem_ld_wait();                                // columns [64 j + 32, 64 j + 64) are in vb
+          if (j + 1 < BN / 64) {
+            tmem_ld32(taddr + (j + 1) * 64, va);
+          } else {
+            // last read of this accumulator: the MMA warp may overwrite it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+              if (leader) mbar_arrive(tempty_bar(acc));
+              else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+            }
+          }
+#if defined(ENTWINE_EXP) && ENTWINE_EXP == 2
+          continue;
+#endif
+          stage32(vb, 1);
+          __syncwarp();
+          // row-wise read-back: eight lanes carry one row's 128 bytes, four rows per instruction
+          uint4 o[8];
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int row = it * 4 + (lane >> 3);
+            o[it] = ld_shared_v4(wstage + row * 128 + (((lane & 7) ^ (row & 7)) << 4));
+          }
+          __syncwarp();  // the staging may be overwritten
+#if !defined(ENTWINE_EXP) || ENTWINE_EXP != 1
+#pragma unroll
+          for (int it = 0; it < 8; ++it)
+            __stcg(reinterpret_cast<uint4*>(cdst + (long long)(it * 4) * P.N + j * 64), o[it]);
+#else
+          if (o[0].x == 0x12345u && o[7].w == 0x54321u) __stcg(reinterpret_cast<uint4*>(cdst), o[0]);
+#endif
+        }
+#endif
+        // the block's stores of this warp are issued; the counter's release orders them before
+        // whatever the flag warp does after it has read the count
+        __syncwarp();
+        if (lane == 0) red_release_cta_add(&sh.warps_stored, 1);
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
+#ifdef ENTWINE_PROFILE
+      if (warp == kEpiWarp0 && lane == 0) prof_acc_[9] += (unsigned long long)(clock64() - prof_epi0);
+#endif
       if (!ok && lane == 0) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -3); }
-    } else if (warp == kCStoreWarp && lane == 0) {
-      // ---- store thread: sends each staged box of the partial C with TMA, returns the staging
-      //      buffers, and counts the blocks whose stores are complete for the flag thread ----
-      int nbox = 0, freed = 0;  // boxes stored / boxes whose staging buffer has been returned
-      int n_issued = 0;         // blocks whose stores are all issued
-      int n_done = 0;           // blocks whose stores are known complete
-      bool ok = true;
-      auto free_upto = [&](int m) {
-        for (; freed <= m; ++freed) mbar_arrive(sfree_bar(freed & 1));
-      };
-      auto mark_done = [&](int n) {
-        if (n == n_done) return;
-        n_done = n;
-        st_release_cta(&sh.blocks_stored, n);
-      };
-      for (int i = 0; ok && i < n_my; ++i) {
-        int d, l;
-        block_of(i, &d, &l);
-        const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
-        for (int j = 0; j < BN / 64; ++j, ++nbox) {
-          const int buf = nbox & 1;
-          if (n_done < n_issued && !mbar_try_wait(staged_bar(buf), (nbox >> 1) & 1)) {
-            // the next box is not staged yet: time to see the issued stores complete
-            bulk_wait_done<0>();
-            free_upto(nbox - 1);
-            mark_done(n_issued);
-          }
-          if (!mbar_wait(staged_bar(buf), (nbox >> 1) & 1, P, &sh)) { ok = false; break; }
-          tma_store_2d(&maps.c_st, nb * BN + j * 64, mb * kBM,
-                       smem_base + n_stages * stage_bytes + buf * kEpiBufBytes);
-          bulk_commit();
-          bulk_wait_read<1>();  // the stores before this one have read their buffers
-          free_upto(nbox - 1);
-          if (n_done < n_issued) {
-            bulk_wait_done<1>();  // all stores but the one just issued, i.e. the earlier blocks'
-            mark_done(n_issued);
-          }
-        }
-        n_issued = i + 1;
-      }
-      bulk_wait_done<0>();
-      if (ok) mark_done(n_issued);
-      else { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -5); }
     } else if (warp == kFlagWarp) {
       // ---- flag warp: releases the tile flags of every block whose stores are complete
       //      (Sec. 4.2).  The release fence takes about a microsecond when memory is busy; in a
@@ -1719,7 +1841,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         int verdict = 0, first = 0, gsize = 1;
         if (lane == 0) {
           for (uint32_t spins = 1; seen <= i; ++spins) {
-            seen = ld_acquire_cta(&sh.blocks_stored);
+            seen = ld_acquire_cta(&sh.warps_stored) / (kEpiThreads / 32);
             if (seen > i) break;
             __nanosleep(64);
             if ((spins % kSpinCheck) == 0) {
@@ -1735,11 +1857,16 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           }
           if (seen > i) {
             t0 = 0;
-            fence_async_all();    // async-proxy writes (the TMA stores) before generic-proxy ones
-            // the stores seen complete by the store thread, then the flags; system scope only
-            // where the flags go to another GPU
-            if (PULL && d != P.r) fence_acq_rel_sys();
-            else fence_acq_rel_gpu();
+            // the epilogue warps' stores (generic-proxy writes, ordered before the count this thread
+            // acquired), then the flags (a consumer that reads the tile with TMA orders its
+            // async-proxy reads after its own acquire); system scope only where the flags go to
+            // another GPU
+            {
+              PROF_T0();
+              if (PULL && d != P.r) fence_acq_rel_sys();
+              else fence_acq_rel_gpu();
+              PROF_ADD(7);
+            }
             if (P.release_group == 1) {
               release_block(d, l);
               verdict = 1;
@@ -1844,8 +1971,13 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   }
 
   // ---------------- exit bookkeeping ----------------
+  PROF_FLUSH(true);
   __syncthreads();
   if (threadIdx.x == 0) atomicMax(&st->t_end, globaltimer_ns());
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const unsigned long long cyc = (unsigned long long)(clock64() - clk0), ns = globaltimer_ns() - ns0;
+    st->clock = (min(cyc, 0xffffffffULL) << 32) | min(ns, 0xffffffffULL);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1871,6 +2003,7 @@ struct DeviceState {
   bool status_pending = false;
   cudaStream_t last_stream = nullptr;
   cudaEvent_t switch_event = nullptr;  // orders a new stream after the plan's last launch
+  unsigned long long last_clock = 0;   // cycles << 32 | ns of CTA 0 in the launch entwine_last_status read
   int64_t withheld = -1;
   // staging for the host-buffer entry point
   cudaStream_t own_stream = nullptr;
@@ -2345,6 +2478,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out);
   kp.cws = (mode == MODE_COMM_ONLY && partial) ? static_cast<const __nv_bfloat16*>(partial) : d->C;
+  kp.cws_out = d->C;
   kp.peers = static_cast<const __nv_bfloat16*>(peers);
   kp.send = static_cast<__nv_bfloat16*>(send);
   kp.flags_own = d->flags_own;
@@ -2499,6 +2633,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   kp.l2_hints = p->l2_hints;
   kp.out = static_cast<__nv_bfloat16*>(out);
   kp.cws = reinterpret_cast<const __nv_bfloat16*>(own_seg + buf_off);
+  kp.cws_out = reinterpret_cast<__nv_bfloat16*>(own_seg + buf_off);
   kp.heap_buf_off = buf_off;
   kp.heap = seg0;
   kp.heap_stride = stride;
@@ -2642,6 +2777,7 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]) {
   out[5] = int64_t(s.tiles_pushed);
   out[6] = (s.t_gemm_end > s.t_start) ? int64_t(s.t_gemm_end - s.t_start) : 0;
   out[7] = (s.t_end > s.t_start) ? int64_t(s.t_end - s.t_start) : 0;
+  d->last_clock = s.clock;
   if (code) {
     // the launch gave up part-way: rewind what its last CTA would have rewound
     cudaMemset(d->list_head, 0, size_t(plan->x + 1) * 2 * 4);
@@ -2651,6 +2787,15 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]) {
     cudaMemcpy(d->status, init, sizeof(init), cudaMemcpyHostToDevice);
   }
   return int(out[0]);
+}
+
+int entwine_last_sm_clock(entwine_plan_t plan, int64_t out[2]) {
+  if (!plan || !out) return ENTWINE_ERR_INVALID;
+  out[0] = out[1] = 0;
+  if (!plan->dev) return ENTWINE_OK;
+  out[0] = int64_t(plan->dev->last_clock >> 32);
+  out[1] = int64_t(plan->dev->last_clock & 0xffffffffULL);
+  return ENTWINE_OK;
 }
 
 int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, const void* peer_partials,
@@ -2883,6 +3028,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
     if (grc != ENTWINE_OK) return grc;
   }
   kp.cws = reinterpret_cast<const __nv_bfloat16*>(base);
+  kp.cws_out = reinterpret_cast<__nv_bfloat16*>(base);
   kp.peers = static_cast<const __nv_bfloat16*>(peer_partials);
   kp.send = static_cast<__nv_bfloat16*>(send_bufs);
   kp.prefetch = p->prefetch;

@@ -36,7 +36,7 @@ SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gem
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
            "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static",
            "entwine_gemm_rs_norm", "entwine_heap_bytes", "entwine_gemm_rs_pull",
-           "entwine_gemm_rs_host_begin", "entwine_gemm_rs_host_wait")
+           "entwine_gemm_rs_host_begin", "entwine_gemm_rs_host_wait", "entwine_last_sm_clock")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
@@ -53,6 +53,7 @@ _lib.entwine_comm_only.argtypes = [_vp, _vp, _vp, _vp, _vp, _int, _vp]
 _lib.entwine_read_partial.argtypes = [_vp, _vp, _vp]
 _lib.entwine_plan_export.argtypes = [_vp, _int, _vp, ctypes.POINTER(ctypes.c_size_t)]
 _lib.entwine_last_status.argtypes = [_vp, ctypes.POINTER(_i64)]
+_lib.entwine_last_sm_clock.argtypes = [_vp, ctypes.POINTER(_i64)]
 _lib.entwine_destroy.argtypes = [_vp]
 _lib.entwine_gemm_rs_static.argtypes = [_vp] * 7 + [ctypes.POINTER(_i64)]
 _lib.entwine_strerror.argtypes = [_int]
@@ -206,6 +207,12 @@ class Plan:
         if check and code != OK:
             raise EntwineError(code, f"device status {st}")
         return st
+
+    def last_sm_clock_mhz(self) -> float:
+        """SM clock of the launch that the last last_status() call reported (0.0 if unknown)."""
+        out = (_i64 * 2)()
+        _check(_lib.entwine_last_sm_clock(self._h, out), "entwine_last_sm_clock")
+        return out[0] / out[1] * 1e3 if out[1] > 0 else 0.0
 
     def destroy(self):
         if self._h:
