@@ -122,6 +122,13 @@ enum {
                                       and >= K_local; 0 (default) = K_local.  May change between
                                       launches                                                     */
   ENTWINE_OPT_LDB             = 17, /* the same for B                                              */
+  ENTWINE_OPT_SPLIT_LAST_WAVE = 19, /* CTA pairs only.  1 (default): when the pair tiles left for the
+                                      last wave occupy at most half of the CTA pairs, each of them is
+                                      computed as two half-width units (256 x 128: one 128 x 128 tile
+                                      per CTA, its flag published by itself) on two pairs, so that
+                                      the last wave costs half a tile time (the producer block may
+                                      be any multiple of the reduction tile, Sec. 4.2); 0: whole
+                                      pair tiles only.  Off with a release group other than 1      */
   ENTWINE_OPT_REG_CONSUMER    = 18, /* how the consumer warps of a CTA that still produces move their
                                       tiles.  1 (default): whole tiles through registers with plain
                                       128-bit loads and stores, so that all shared memory and the

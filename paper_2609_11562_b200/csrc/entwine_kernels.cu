@@ -124,6 +124,9 @@ struct KParams {
   int prefetch;   // pull the next reduce task's peer tiles into L2 ahead of its loads
   int l2_hints;   // consumer TMA traffic carries an evict-first L2 policy
   int stages;     // operand-ring stages of the producer
+  int split;      // pair tiles: the last `split` pair tiles of the order are each done as two half-width
+                  // units (256 x 128: one 128 x 128 tile per CTA), so that a last wave that fills at
+                  // most half of the CTA pairs costs half a tile time; 0 = none
   int kpb;        // k-blocks (64 elements of K) per stage
   int k3d;        // 1: a stage's k-blocks of one operand arrive as ONE 3-D TMA box (the SM's TMA unit keeps
                   // only about two load instructions in flight, so bytes per instruction bound its rate)
@@ -183,6 +186,7 @@ struct KParams {
 struct KMaps {
   CUtensorMap a, b;      // operands, one k-block per box
   CUtensorMap a3, b3;    // operands viewed as [K/64][rows][64]: one box brings kpb k-blocks (k3d)
+  CUtensorMap bh, bh3;   // B with boxes of 64 rows: a CTA's share of a half-width pair tile
   CUtensorMap c_st;      // partial C, box 64 x 128, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
@@ -1466,7 +1470,9 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
   const bool leader = cta_rank == 0;
   // work units of a producer: blocks p = g, g+G, ... or, for pairs, pair indices u = g/2, ...
-  const int n_units = PAIR ? P.P_blk / 2 : P.P_blk;
+  // (with a split last wave the last P.split pair tiles count as two units each)
+  const int n_full = PAIR ? P.P_blk / 2 - P.split : P.P_blk;
+  const int n_units = n_full + (PAIR ? 2 * P.split : 0);
   const int unit0 = PAIR ? g / 2 : g;
   const int stride = PAIR ? P.G / 2 : P.G;
   const int n_my = (is_producer && unit0 < n_units) ? (n_units - unit0 + stride - 1) / stride : 0;
@@ -1550,8 +1556,14 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
     const int KB = (P.K + kBK - 1) / kBK;
     // block i of this CTA: its position in the tile order (returned), its destination partition
     // d and its index l inside the partition
-    auto block_of = [&](int i, int* d, int* l) {
-      const int unit = unit0 + i * stride;
+    // *half: -1 for a whole block; 0 / 1 when this unit is the left / right 128 columns of it
+    auto block_of = [&](int i, int* d, int* l, int* half) {
+      int unit = unit0 + i * stride;
+      *half = -1;
+      if (PAIR && unit >= n_full) {
+        *half = (unit - n_full) & 1;
+        unit = n_full + ((unit - n_full) >> 1);
+      }
       const int p = PAIR ? pair_position(P, unit, (int)cta_rank) : unit;
       position_to_block(P, p, d, l);
       return p;
@@ -1565,10 +1577,15 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       uint32_t phase = 0;
       bool ok = true;
       for (int i = 0; ok && i < n_my; ++i) {
-        int d, l;
-        block_of(i, &d, &l);
+        int d, l, half;
+        block_of(i, &d, &l, &half);
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
-        const int b_row = nb * BN + (PAIR ? (int)cta_rank * C::kBRows : 0);
+        // rows of B this CTA loads: its half of the block's columns, or of the half block's
+        const int b_rows = half < 0 ? C::kBRows : C::kBRows / 2;
+        const int b_row = nb * BN + (half < 0 ? 0 : half * (BN / 2)) + (PAIR ? (int)cta_rank * b_rows : 0);
+        const int b_bytes = b_rows * kBK * 2;  // one k-block of them
+        const CUtensorMap* const mb2 = half < 0 ? &maps.b : &maps.bh;
+        const CUtensorMap* const mb3 = half < 0 ? &maps.b3 : &maps.bh3;
         for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
           {
             PROF_T0();
@@ -1585,17 +1602,17 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
             // one box per operand: [kpb k-blocks][rows][64]; k-blocks past the end of K read as zero
             if (PAIR) {
               // both CTAs' bytes are counted on the leader's barrier, which the leader arms
-              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * stage_bytes);
+              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * P.kpb * (C::kABytes + b_bytes));
               tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
-              tma_load_3d_pair_hint(b_dst, &maps.b3, 0, b_row, kb0, lead_bar, op_pol);
+              tma_load_3d_pair_hint(b_dst, mb3, 0, b_row, kb0, lead_bar, op_pol);
             } else {
               mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
               tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, full_bar(stage), op_pol);
-              tma_load_3d_hint(b_dst, &maps.b3, 0, b_row, kb0, full_bar(stage), op_pol);
+              tma_load_3d_hint(b_dst, mb3, 0, b_row, kb0, full_bar(stage), op_pol);
             }
           } else {
             if (PAIR) {
-              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * nkb * C::kKBlockBytes);
+              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * nkb * (C::kABytes + b_bytes));
             } else {
               mbar_arrive_expect_tx(full_bar(stage), nkb * C::kKBlockBytes);
             }
@@ -1603,7 +1620,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
               const int kx = (kb0 + kk) * kBK;
               if (PAIR) {
                 tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, lead_bar, op_pol);
-                tma_load_2d_pair_hint(b_dst + kk * C::kBBytes, &maps.b, kx, b_row, lead_bar, op_pol);
+                tma_load_2d_pair_hint(b_dst + kk * b_bytes, mb2, kx, b_row, lead_bar, op_pol);
               } else {
                 tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, full_bar(stage), op_pol);
                 tma_load_2d_hint(b_dst + kk * C::kBBytes, &maps.b, kx, b_row, full_bar(stage), op_pol);
@@ -1620,12 +1637,17 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
-      constexpr uint32_t idesc = instr_desc<BN, PAIR ? 256 : 128>();
+      constexpr uint32_t idesc_full = instr_desc<BN, PAIR ? 256 : 128>();
+      constexpr uint32_t idesc_half = instr_desc<BN / 2, PAIR ? 256 : 128>();
       bool ok = true;
 #ifdef ENTWINE_PROFILE
       const long long prof_mma0 = clock64();
 #endif
       for (int i = 0; ok && i < n_my; ++i) {
+        int d_, l_, half;
+        block_of(i, &d_, &l_, &half);
+        const uint32_t idesc = half < 0 ? idesc_full : idesc_half;
+        const int b_bytes = (half < 0 ? C::kBRows : C::kBRows / 2) * kBK * 2;
         {
           PROF_T0();
           const bool got = mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh);
@@ -1647,7 +1669,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           const int nkb = min(P.kpb, KB - kb0);
           for (int kk = 0; kk < nkb; ++kk) {
             const uint64_t a_desc = smem_desc_sw128(a_s + kk * C::kABytes);
-            const uint64_t b_desc = smem_desc_sw128(b_s + kk * C::kBBytes);
+            const uint64_t b_desc = smem_desc_sw128(b_s + kk * b_bytes);
 #pragma unroll
             for (int k = 0; k < kBK / kUmmaK; ++k) {
               // advancing K by 16 elements = 32 bytes = 2 descriptor address units
@@ -1687,9 +1709,11 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       const long long prof_epi0 = clock64();
 #endif
       for (int i = 0; ok && i < n_my; ++i) {
-        int d, l;
-        block_of(i, &d, &l);
+        int d, l, half;
+        block_of(i, &d, &l, &half);
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
+        const int n_cols64 = half < 0 ? BN / 64 : BN / 128;        // 64-column units of this unit
+        const int col0 = nb * BN + (half < 0 ? 0 : half * (BN / 2));
         {
           PROF_T0();
           ok = mbar_wait(tfull_bar(acc), acc_phase, P, &sh);
@@ -1705,7 +1729,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         }
         const uint32_t taddr = tmem_base + (uint32_t(q * 32) << 16) + acc * BN;
         // this lane's share of a read-back: row (lane / 8) + 4 * it of the warp's 32, 16-byte chunk lane % 8
-        __nv_bfloat16* const cdst = P.cws_out + (long long)(mb * kBM + q * 32 + (lane >> 3)) * P.N + nb * BN + (lane & 7) * 8;
+        __nv_bfloat16* const cdst = P.cws_out + (long long)(mb * kBM + q * 32 + (lane >> 3)) * P.N + col0 + (lane & 7) * 8;
         // Two register sets: the TMEM load of the next 32 columns is in flight while the previous
         // 32 are rounded and staged (a tcgen05.ld takes a few hundred cycles).
         uint32_t va[32], vb[32];
@@ -1726,53 +1750,14 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
             st_shared_v4(my_row + ((chunk ^ (lane & 7)) << 4), o);
           }
         };
-#if defined(ENTWINE_EXP) && ENTWINE_EXP == 3
-        // each lane writes its own row: 64 bytes per 32 columns, as four 16-byte stores
-        __nv_bfloat16* const crow = P.cws_out + (long long)(mb * kBM + q * 32 + lane) * P.N + nb * BN;
-        auto direct32 = [&](const uint32_t (&v)[32], int col) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            uint4 o;
-            uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(v[8 * e + 2 * u]),
-                                                        __uint_as_float(v[8 * e + 2 * u + 1]));
-              ow[u] = *reinterpret_cast<uint32_t*>(&hh);
-            }
-            __stcg(reinterpret_cast<uint4*>(crow + col + e * 8), o);
-          }
-        };
         tmem_ld32(taddr, va);
 #pragma unroll 1
-        for (int j = 0; j < BN / 64; ++j) {
-          tmem_ld_wait();
-          tmem_ld32(taddr + j * 64 + 32, vb);
-          direct32(va, j * 64);
-          tmem_ld_wait();
-          if (j + 1 < BN / 64) {
-            tmem_ld32(taddr + (j + 1) * 64, va);
-          } else {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-              if (leader) mbar_arrive(tempty_bar(acc));
-              else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
-            }
-          }
-          direct32(vb, j * 64 + 32);
-        }
-#else
-        tmem_ld32(taddr, va);
-#pragma unroll 1
-        for (int j = 0; j < BN / 64; ++j) {
+        for (int j = 0; j < n_cols64; ++j) {
           tmem_ld_wait();                                // columns [64 j, 64 j + 32) are in va
           tmem_ld32(taddr + j * 64 + 32, vb);
-#if !defined(ENTWINE_EXP) || ENTWINE_EXP != 2
           stage32(va, 0);
-#endif
           tmem_ld_wait();                                // columns [64 j + 32, 64 j + 64) are in vb
-          if (j + 1 < BN / 64) {
+          if (j + 1 < n_cols64) {
             tmem_ld32(taddr + (j + 1) * 64, va);
           } else {
             // last read of this accumulator: the MMA warp may overwrite it
@@ -1783,9 +1768,6 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
               else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
             }
           }
-#if defined(ENTWINE_EXP) && ENTWINE_EXP == 2
-          continue;
-#endif
           stage32(vb, 1);
           __syncwarp();
           // row-wise read-back: eight lanes carry one row's 128 bytes, four rows per instruction
@@ -1796,15 +1778,10 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
             o[it] = ld_shared_v4(wstage + row * 128 + (((lane & 7) ^ (row & 7)) << 4));
           }
           __syncwarp();  // the staging may be overwritten
-#if !defined(ENTWINE_EXP) || ENTWINE_EXP != 1
 #pragma unroll
           for (int it = 0; it < 8; ++it)
             __stcg(reinterpret_cast<uint4*>(cdst + (long long)(it * 4) * P.N + j * 64), o[it]);
-#else
-          if (o[0].x == 0x12345u && o[7].w == 0x54321u) __stcg(reinterpret_cast<uint4*>(cdst), o[0]);
-#endif
         }
-#endif
         // the block's stores of this warp are issued; the counter's release orders them before
         // whatever the flag warp does after it has read the count
         __syncwarp();
@@ -1822,20 +1799,22 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       //      counts; a group release (the granularity ablation) is spread over the lanes ----
       int seen = 0;
       unsigned long long t0 = 0;
-      auto release_block = [&](int dd, int ll) {
-        const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb;
+      // half < 0: all tiles of the block; else the one tile a half-width unit covers
+      auto release_block = [&](int dd, int ll, int half) {
+        const int t_first = (ll / P.nBn) * P.nTn + (ll % P.nBn) * P.cpb + (half < 0 ? 0 : half);
+        const int n_t = half < 0 ? P.cpb : 1;
         if (PULL && dd != P.r) {
           // the flag goes to its reader: row r of destination dd's flag array
           unsigned* f = reinterpret_cast<unsigned*>(P.heap + dd * P.heap_stride + P.heap_flags_off) + P.r * P.Q;
-          for (int c = 0; c < P.cpb; ++c) st_relaxed_sys(&f[t_first + c], P.epoch);
+          for (int c = 0; c < n_t; ++c) st_relaxed_sys(&f[t_first + c], P.epoch);
         } else {
-          for (int c = 0; c < P.cpb; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
+          for (int c = 0; c < n_t; ++c) st_relaxed_gpu(&P.flags_own[dd * P.Q + t_first + c], P.epoch);
         }
-        published += P.cpb;
+        published += n_t;
       };
       for (int i = 0; i < n_my; ++i) {
-        int d, l;
-        const int pos = block_of(i, &d, &l);
+        int d, l, half;
+        const int pos = block_of(i, &d, &l, &half);
         // what lane 0 finds: 0 = stop (abort / timeout), 1 = nothing to release for this block,
         // 2 = release the group [first, first + gsize) (or partition d)
         int verdict = 0, first = 0, gsize = 1;
@@ -1868,7 +1847,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
               PROF_ADD(7);
             }
             if (P.release_group == 1) {
-              release_block(d, l);
+              release_block(d, l, half);
               verdict = 1;
             } else {
               // Coarser release: the block is counted in its group; whoever stores a group's
@@ -1895,11 +1874,11 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         fence_acq_rel_gpu();  // the other blocks' stores, released by their CTAs' counts
         for (int j = lane; j < gsize; j += 32) {
           if (P.release_group == ENTWINE_RELEASE_PARTITION) {
-            release_block(d, j);
+            release_block(d, j, -1);
           } else {
             int dd, ll;
             position_to_block(P, first + j, &dd, &ll);
-            release_block(dd, ll);
+            release_block(dd, ll, -1);
           }
         }
       }
@@ -2078,20 +2057,22 @@ static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_
 static bool make_operand_maps(KMaps* maps, const void* A, const void* B, const Geometry& g, int b_rows, int kpb,
                               int64_t lda, int64_t ldb, int* k3d) {
   *k3d = 0;
-  if (!make_map(&maps->a, A, g.M, g.K, kBK, kBM, true, lda) || !make_map(&maps->b, B, g.N, g.K, kBK, b_rows, true, ldb))
+  // (bh, bh3: half as many rows of B per box, for the half-width units of a split last wave)
+  if (!make_map(&maps->a, A, g.M, g.K, kBK, kBM, true, lda) || !make_map(&maps->b, B, g.N, g.K, kBK, b_rows, true, ldb) ||
+      !make_map(&maps->bh, B, g.N, g.K, kBK, b_rows / 2, true, ldb))
     return false;
   if (kpb < 2 || g.K % kBK != 0) return true;
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   bool ok = true;
-  for (int op = 0; op < 2; ++op) {
+  for (int op = 0; op < 3; ++op) {
     const int64_t rows = op == 0 ? g.M : g.N;
     const int64_t ld = op == 0 ? (lda > 0 ? lda : g.K) : (ldb > 0 ? ldb : g.K);
     cuuint64_t dims[3] = {cuuint64_t(kBK), cuuint64_t(rows), cuuint64_t(g.K / kBK)};
     cuuint64_t strides[2] = {cuuint64_t(ld) * 2, cuuint64_t(kBK) * 2};
-    cuuint32_t box[3] = {cuuint32_t(kBK), cuuint32_t(op == 0 ? kBM : b_rows), cuuint32_t(kpb)};
+    cuuint32_t box[3] = {cuuint32_t(kBK), cuuint32_t(op == 0 ? kBM : (op == 1 ? b_rows : b_rows / 2)), cuuint32_t(kpb)};
     cuuint32_t estr[3] = {1, 1, 1};
-    CUresult rc = fn(op == 0 ? &maps->a3 : &maps->b3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+    CUresult rc = fn(op == 0 ? &maps->a3 : (op == 1 ? &maps->b3 : &maps->bh3), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
                      const_cast<void*>(op == 0 ? A : B), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -2099,6 +2080,17 @@ static bool make_operand_maps(KMaps* maps, const void* A, const void* B, const G
   }
   *k3d = ok ? 1 : 0;  // without them a stage is filled k-block by k-block
   return true;
+}
+
+// Split last wave (CTA pairs only): if the pair tiles left over after the last full wave occupy at
+// most half of the n_pairs CTA pairs, each of them is done as two half-width units on two pairs, and
+// the last wave costs half a tile time.  Returns how many pair tiles are split.
+static int split_last_wave(const Plan* p, int n_producer_ctas) {
+  if (!p->pair || !p->split_opt || p->release_group != 1) return 0;
+  const int n_pairs = n_producer_ctas / 2, n_tiles = p->g.P_blk / 2;
+  if (n_pairs < 1) return 0;
+  const int rest = n_tiles % n_pairs;
+  return (rest > 0 && 2 * rest <= n_pairs) ? rest : 0;
 }
 
 // Tasks per claim: as many as have their flags (W per reduce task) in the 64 flag values the
@@ -2512,6 +2504,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
     else grid += 1, kp.n_ded += 1;
     if (kp.n_ded < p->x) kp.help = 1;
   }
+  kp.split = (mode != MODE_COMM_ONLY) ? split_last_wave(p, kp.G) : 0;
 
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
@@ -2660,6 +2653,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
     else grid += 1, kp.n_ded += 1;
     if (kp.n_ded < p->x) kp.help = 1;
   }
+  kp.split = split_last_wave(p, kp.G);
 
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
@@ -3051,6 +3045,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
     else grid += 1, kp.n_ded += 1;
     if (kp.n_ded < p->x) kp.help = 1;
   }
+  kp.split = split_last_wave(p, kp.G);
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d) &&

@@ -280,6 +280,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);
       return ENTWINE_OK;
+    case ENTWINE_OPT_SPLIT_LAST_WAVE:
+      if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
+      p->split_opt = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_REG_CONSUMER:
       if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
       p->reg_consumer = int(value);
