@@ -179,6 +179,26 @@ enum {
 int entwine_plan(entwine_plan_t* plan, int64_t M, int64_t N, int64_t K_local, int W,
                  int tile_order, int n_comm_sms);
 
+/*
+ * entwine_plan_workspace_bytes / entwine_plan_set_workspace - let the caller's allocator own the
+ * plan's device memory.  Without these calls the plan allocates its arrays with cudaMalloc at the
+ * first call that needs the device; with them, everything the plan (and its layer-chain and
+ * pull-mode calls) would allocate lives in one caller-provided block.
+ *   _workspace_bytes  writes the size of that block for the plan as it is now ([pre] options
+ *                     that change the tables change the size: query after setting them).
+ *   _set_workspace    workspace: device pointer, 256-byte aligned, at least that size, valid until
+ *                     entwine_destroy (the library never frees it); NULL returns the plan to
+ *                     memory of its own.  The call initialises the block (synchronous copies of
+ *                     the task tables, cleared flags and status) and performs the per-device
+ *                     kernel set-up, so the plan's first launch neither allocates nor
+ *                     synchronises and may already be captured into a CUDA graph.
+ * Call before the plan's first launch.  Errors: ENTWINE_ERR_INVALID (after a launch, misaligned
+ * or too small), ENTWINE_ERR_RESOURCES, ENTWINE_ERR_CUDA.  A [pre] option set afterwards keeps
+ * the block; the next call fails with ENTWINE_ERR_INVALID if the rebuilt tables no longer fit it.
+ */
+int entwine_plan_workspace_bytes(entwine_plan_t plan, size_t* bytes);
+int entwine_plan_set_workspace(entwine_plan_t plan, void* workspace, size_t bytes);
+
 /* entwine_set_option - see ENTWINE_OPT_*.  Errors: ENTWINE_ERR_INVALID (unknown key, bad
  * value, or a [pre] option after the first launch). */
 int entwine_set_option(entwine_plan_t plan, int key, int64_t value);

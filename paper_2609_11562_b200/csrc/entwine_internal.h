@@ -97,6 +97,8 @@ struct Plan {
   int n_gemm_ctas = 0;  // producer CTAs of the fused launch
   int n_comm_ctas = 0;  // dedicated consumer CTAs of the fused launch
   HostTables tables;
+  void* ws_ptr = nullptr;   // caller-provided device workspace (entwine_plan_set_workspace), or null
+  size_t ws_bytes = 0;
   DeviceState* dev = nullptr;
 };
 

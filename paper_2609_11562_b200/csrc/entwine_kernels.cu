@@ -1978,6 +1978,7 @@ struct DeviceState {
   unsigned* band_ctr = nullptr;  // layer chain: [rowsT]
   unsigned epoch = 0;
   unsigned seq = 0;
+  bool user_ws = false;   // the arrays below live in the caller's workspace (nothing of them is freed here)
   bool captured = false;  // a launch of this plan has been captured into a CUDA graph
   bool status_pending = false;
   cudaStream_t last_stream = nullptr;
@@ -2121,6 +2122,37 @@ int device_sm_count() {
     }                                      \
   } while (0)
 
+// Plan-owned device memory: one section per array, each starting on a 256-byte boundary.  The same
+// layout serves cudaMalloc'ed arrays (one allocation each) and a caller-provided workspace (one
+// block, entwine_plan_set_workspace), which also holds what the layer chain and the pull mode
+// would otherwise allocate at their first call.
+struct WorkspaceLayout {
+  size_t c, flags_own, flags_peer, tasks, list_offs, list_head, status, group_ctr, ssq_part, band_ctr, tasks_pull,
+      list_offs_pull, total;
+};
+static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
+static WorkspaceLayout workspace_layout(const Plan* p) {
+  const Geometry& g = p->g;
+  const HostTables& t = p->tables;
+  WorkspaceLayout w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += align256(std::max<size_t>(bytes, 1)); return at; };
+  w.c = take(size_t(g.M) * g.N * 2);
+  w.flags_own = take(size_t(g.W) * g.Q * 4);
+  w.flags_peer = take(size_t(g.W - 1) * g.Q * 4);
+  w.tasks = take(t.dev_tasks.size() * sizeof(Task));
+  w.list_offs = take(t.list_offs.size() * 4);
+  w.list_head = take(size_t(p->x + 1) * 2 * 4);
+  w.status = take(2 * sizeof(StatusSlot));
+  w.group_ctr = take(size_t(g.P_blk) * 4);
+  w.ssq_part = take(size_t(g.R) * g.nTn * 4);
+  w.band_ctr = take(size_t(g.rowsT) * 4);
+  w.tasks_pull = take(t.pull_tasks.size() * sizeof(Task));
+  w.list_offs_pull = take(t.pull_list_offs.size() * 4);
+  w.total = off;
+  return w;
+}
+
 static int ensure_device(Plan* p) {
   if (p->dev) return ENTWINE_OK;
   int sms = device_sm_count();
@@ -2131,19 +2163,43 @@ static int ensure_device(Plan* p) {
   CK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
   if (major != 10) return ENTWINE_ERR_RESOURCES;  // tcgen05 / TMEM needed
   if (p->num_sms > sms) return ENTWINE_ERR_RESOURCES;
+  const WorkspaceLayout w = workspace_layout(p);
+  if (p->ws_ptr && p->ws_bytes < w.total) return ENTWINE_ERR_INVALID;  // the tables grew after set_workspace
   DeviceState* d = new DeviceState();
   d->device = dev;
   const Geometry& g = p->g;
   const size_t n_own = size_t(g.W) * g.Q, n_peer = size_t(g.W - 1) * g.Q;
   const HostTables& t = p->tables;
-  bool ok = cudaMalloc(&d->C, size_t(g.M) * g.N * 2) == cudaSuccess &&
-            cudaMalloc(&d->flags_own, n_own * 4) == cudaSuccess &&
-            cudaMalloc(&d->flags_peer, n_peer * 4) == cudaSuccess &&
-            cudaMalloc(&d->tasks, t.dev_tasks.size() * sizeof(Task)) == cudaSuccess &&
-            cudaMalloc(&d->list_offs, t.list_offs.size() * 4) == cudaSuccess &&
-            cudaMalloc(&d->list_head, size_t(p->x + 1) * 2 * 4) == cudaSuccess &&
-            cudaMalloc(&d->status, 2 * sizeof(StatusSlot)) == cudaSuccess &&
-            cudaMalloc(&d->group_ctr, size_t(g.P_blk) * 4) == cudaSuccess;
+  bool ok;
+  if (p->ws_ptr) {
+    char* b = static_cast<char*>(p->ws_ptr);
+    d->user_ws = true;
+    d->C = reinterpret_cast<__nv_bfloat16*>(b + w.c);
+    d->flags_own = reinterpret_cast<unsigned*>(b + w.flags_own);
+    d->flags_peer = reinterpret_cast<unsigned*>(b + w.flags_peer);
+    d->tasks = reinterpret_cast<Task*>(b + w.tasks);
+    d->list_offs = reinterpret_cast<int*>(b + w.list_offs);
+    d->list_head = reinterpret_cast<int*>(b + w.list_head);
+    d->status = reinterpret_cast<StatusSlot*>(b + w.status);
+    d->group_ctr = reinterpret_cast<unsigned*>(b + w.group_ctr);
+    d->ssq_part = reinterpret_cast<float*>(b + w.ssq_part);
+    d->band_ctr = reinterpret_cast<unsigned*>(b + w.band_ctr);
+    d->tasks_pull = reinterpret_cast<Task*>(b + w.tasks_pull);
+    d->list_offs_pull = reinterpret_cast<int*>(b + w.list_offs_pull);
+    ok = cudaMemcpy(d->tasks_pull, t.pull_tasks.data(), t.pull_tasks.size() * sizeof(Task), cudaMemcpyHostToDevice) ==
+             cudaSuccess &&
+         cudaMemcpy(d->list_offs_pull, t.pull_list_offs.data(), t.pull_list_offs.size() * 4, cudaMemcpyHostToDevice) ==
+             cudaSuccess;
+  } else {
+    ok = cudaMalloc(&d->C, size_t(g.M) * g.N * 2) == cudaSuccess &&
+         cudaMalloc(&d->flags_own, n_own * 4) == cudaSuccess &&
+         cudaMalloc(&d->flags_peer, n_peer * 4) == cudaSuccess &&
+         cudaMalloc(&d->tasks, t.dev_tasks.size() * sizeof(Task)) == cudaSuccess &&
+         cudaMalloc(&d->list_offs, t.list_offs.size() * 4) == cudaSuccess &&
+         cudaMalloc(&d->list_head, size_t(p->x + 1) * 2 * 4) == cudaSuccess &&
+         cudaMalloc(&d->status, 2 * sizeof(StatusSlot)) == cudaSuccess &&
+         cudaMalloc(&d->group_ctr, size_t(g.P_blk) * 4) == cudaSuccess;
+  }
   if (ok) {
     StatusSlot init[2];
     std::memset(init, 0, sizeof(init));
@@ -2198,18 +2254,20 @@ void device_release(Plan* p) {
     cudaStreamDestroy(d->own_stream);
   }
   if (d->switch_event) cudaEventDestroy(d->switch_event);
-  cudaFree(d->C);
-  cudaFree(d->flags_own);
-  cudaFree(d->flags_peer);
-  cudaFree(d->tasks);
-  cudaFree(d->list_offs);
-  cudaFree(d->list_head);
-  cudaFree(d->status);
-  cudaFree(d->group_ctr);
-  cudaFree(d->tasks_pull);
-  cudaFree(d->list_offs_pull);
-  cudaFree(d->ssq_part);
-  cudaFree(d->band_ctr);
+  if (!d->user_ws) {
+    cudaFree(d->C);
+    cudaFree(d->flags_own);
+    cudaFree(d->flags_peer);
+    cudaFree(d->tasks);
+    cudaFree(d->list_offs);
+    cudaFree(d->list_head);
+    cudaFree(d->status);
+    cudaFree(d->group_ctr);
+    cudaFree(d->tasks_pull);
+    cudaFree(d->list_offs_pull);
+    cudaFree(d->ssq_part);
+    cudaFree(d->band_ctr);
+  }
   cudaFree(d->sA);
   cudaFree(d->sB);
   cudaFree(d->sPeers);
@@ -2235,8 +2293,9 @@ static cudaError_t order_after_last_launch(DeviceState* d, cudaStream_t stream) 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 template <int BN, bool PAIR, bool NORM = false, bool PULL = false>
-static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream) {
-  if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false>(p, kp, maps, grid, stream);
+static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream,
+                     bool config_only = false) {
+  if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false>(p, kp, maps, grid, stream, config_only);
   // per device: the shared-memory opt-in has been set, and how many clusters fit at once (shared by
   // all plans, which may be used from different threads)
   static int max_clusters[64] = {0};
@@ -2259,18 +2318,23 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  std::lock_guard<std::mutex> lock(config_mutex);
-  if (!configured[dev]) {
-    CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    int per_sm = 0;
-    CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
-    if (per_sm < 1) return ENTWINE_ERR_RESOURCES;
-    if (PAIR) CK(cudaOccupancyMaxActiveClusters(&max_clusters[dev], kern, &cfg));
-    configured[dev] = true;
+  int clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(config_mutex);
+    if (!configured[dev]) {
+      CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+      int per_sm = 0;
+      CK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, kSmemBytes));
+      if (per_sm < 1) return ENTWINE_ERR_RESOURCES;
+      if (PAIR) CK(cudaOccupancyMaxActiveClusters(&max_clusters[dev], kern, &cfg));
+      configured[dev] = true;
+    }
+    clusters = max_clusters[dev];
   }
   // every cluster of the grid must be resident at once: producers and consumers wait on each
   // other inside one launch
-  if (PAIR && max_clusters[dev] * 2 < grid) return ENTWINE_ERR_RESOURCES;
+  if (PAIR && clusters * 2 < grid) return ENTWINE_ERR_RESOURCES;
+  if (config_only) return ENTWINE_OK;
   CK(cudaLaunchKernelEx(&cfg, kern, maps, kp));
   CK(cudaGetLastError());
   return ENTWINE_OK;
@@ -2350,8 +2414,9 @@ struct NormArgs {
 
 static int launch(Plan* p, int mode, const void* A, const void* B, const void* partial, const void* peers,
                   void* out, void* send, int n_ctas, cudaStream_t stream, const NormArgs* norm = nullptr) {
-  if (!p->dev || !p->launched) {
+  if (!p->dev || !(p->launched || p->dev->user_ws)) {
     // the first launch allocates the workspace and configures the kernel: not inside a capture
+    // (a plan with a caller-provided workspace did both in entwine_plan_set_workspace)
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) {
       cudaGetLastError();
@@ -2394,7 +2459,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   CK(cudaStreamIsCapturing(stream, &cap));
   const bool capturing = cap != cudaStreamCaptureStatusNone;
   if (capturing) {
-    if (!p->launched || (norm && !d->ssq_part)) return ENTWINE_ERR_INVALID;
+    if (!(p->launched || d->user_ws) || (norm && !d->ssq_part)) return ENTWINE_ERR_INVALID;
     d->captured = true;
   }
 
@@ -2783,6 +2848,52 @@ int entwine_last_status(entwine_plan_t plan, int64_t out[8]) {
   return int(out[0]);
 }
 
+int entwine_plan_workspace_bytes(entwine_plan_t plan, size_t* bytes) {
+  if (!plan || !bytes) return ENTWINE_ERR_INVALID;
+  *bytes = workspace_layout(plan).total;
+  return ENTWINE_OK;
+}
+
+int entwine_plan_set_workspace(entwine_plan_t plan, void* workspace, size_t bytes) {
+  if (!plan || plan->launched) return ENTWINE_ERR_INVALID;
+  Plan* p = plan;
+  if (p->dev) device_release(p);
+  p->ws_ptr = nullptr;
+  p->ws_bytes = 0;
+  if (!workspace) return ENTWINE_OK;  // back to memory of the library's own
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) || bytes < workspace_layout(p).total) return ENTWINE_ERR_INVALID;
+  p->ws_ptr = workspace;
+  p->ws_bytes = bytes;
+  int rc = ensure_device(p);  // carves the block and fills tables, flags and status (synchronous copies)
+  if (rc == ENTWINE_OK) {
+    // everything else a first launch would do once per device: the kernels' shared-memory opt-in
+    // and the residency check, for every variant this plan can launch
+    KParams kp;
+    std::memset(&kp, 0, sizeof(kp));
+    KMaps maps;
+    std::memset(&maps, 0, sizeof(maps));
+    const int grid = std::min(p->num_sms, p->n_gemm_ctas + p->n_comm_ctas);
+    for (int variant = 0; rc == ENTWINE_OK && variant < 3; ++variant) {
+      kp.norm = variant == 1;
+      if (variant == 2) {
+        if (p->pair) rc = launch_bn<256, true, false, true>(p, kp, maps, grid, nullptr, true);
+        else if (p->g.BN == 256) rc = launch_bn<256, false, false, true>(p, kp, maps, grid, nullptr, true);
+        else rc = launch_bn<128, false, false, true>(p, kp, maps, grid, nullptr, true);
+      } else {
+        if (p->pair) rc = launch_bn<256, true>(p, kp, maps, grid, nullptr, true);
+        else if (p->g.BN == 256) rc = launch_bn<256, false>(p, kp, maps, grid, nullptr, true);
+        else rc = launch_bn<128, false>(p, kp, maps, grid, nullptr, true);
+      }
+    }
+  }
+  if (rc != ENTWINE_OK) {
+    if (p->dev) device_release(p);
+    p->ws_ptr = nullptr;
+    p->ws_bytes = 0;
+  }
+  return rc;
+}
+
 int entwine_last_sm_clock(entwine_plan_t plan, int64_t out[2]) {
   if (!plan || !out) return ENTWINE_ERR_INVALID;
   out[0] = out[1] = 0;
@@ -2931,8 +3042,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartialMa
 // stand-in for the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
 constexpr int kMaxDevices = 64;
 static unsigned char* g_static_scratch_addr[kMaxDevices] = {nullptr};
-
-static size_t align256(size_t v) { return (v + 255) / 256 * 256; }
 
 }  // namespace entwine
 

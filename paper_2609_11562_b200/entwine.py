@@ -36,7 +36,8 @@ SYMBOLS = ("entwine_plan", "entwine_set_option", "entwine_gemm_rs", "entwine_gem
            "entwine_gemm_only", "entwine_comm_only", "entwine_read_partial", "entwine_plan_export",
            "entwine_last_status", "entwine_destroy", "entwine_strerror", "entwine_gemm_rs_static",
            "entwine_gemm_rs_norm", "entwine_heap_bytes", "entwine_gemm_rs_pull",
-           "entwine_gemm_rs_host_begin", "entwine_gemm_rs_host_wait", "entwine_last_sm_clock")
+           "entwine_gemm_rs_host_begin", "entwine_gemm_rs_host_wait", "entwine_last_sm_clock",
+           "entwine_plan_workspace_bytes", "entwine_plan_set_workspace")
 
 _vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
 _lib.entwine_plan.argtypes = [ctypes.POINTER(_vp), _i64, _i64, _i64, _int, _int, _int]
@@ -54,6 +55,8 @@ _lib.entwine_read_partial.argtypes = [_vp, _vp, _vp]
 _lib.entwine_plan_export.argtypes = [_vp, _int, _vp, ctypes.POINTER(ctypes.c_size_t)]
 _lib.entwine_last_status.argtypes = [_vp, ctypes.POINTER(_i64)]
 _lib.entwine_last_sm_clock.argtypes = [_vp, ctypes.POINTER(_i64)]
+_lib.entwine_plan_workspace_bytes.argtypes = [_vp, ctypes.POINTER(ctypes.c_size_t)]
+_lib.entwine_plan_set_workspace.argtypes = [_vp, _vp, ctypes.c_size_t]
 _lib.entwine_destroy.argtypes = [_vp]
 _lib.entwine_gemm_rs_static.argtypes = [_vp] * 7 + [ctypes.POINTER(_i64)]
 _lib.entwine_strerror.argtypes = [_int]
@@ -208,10 +211,26 @@ class Plan:
             raise EntwineError(code, f"device status {st}")
         return st
 
+    def workspace_bytes(self) -> int:
+        n = ctypes.c_size_t(0)
+        _check(_lib.entwine_plan_workspace_bytes(self._h, ctypes.byref(n)), "entwine_plan_workspace_bytes")
+        return int(n.value)
+
+    def set_workspace(self, buf, nbytes=None):
+        """buf: a CUDA tensor (kept alive by this object) or a raw device address with nbytes."""
+        if buf is None:
+            _check(_lib.entwine_plan_set_workspace(self._h, None, 0), "entwine_plan_set_workspace")
+            self._ws = None
+            return
+        n = nbytes if nbytes is not None else buf.numel() * buf.element_size()
+        _check(_lib.entwine_plan_set_workspace(self._h, _ptr(buf), n), "entwine_plan_set_workspace")
+        self._ws = buf
+
     def last_sm_clock_mhz(self) -> float:
         """SM clock of the launch that the last last_status() call reported (0.0 if unknown)."""
         out = (_i64 * 2)()
-        _check(_lib.entwine_last_sm_clock(self._h, out), "entwine_last_sm_clock")
+        _check(_lib.entwine_last_sm_clock(self._h, out), "entwine_last_sm_clock",
+           "entwine_plan_workspace_bytes", "entwine_plan_set_workspace")
         return out[0] / out[1] * 1e3 if out[1] > 0 else 0.0
 
     def destroy(self):

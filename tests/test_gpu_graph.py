@@ -97,3 +97,59 @@ def test_capture_before_the_first_launch_is_refused():
                 plan.gemm_rs(A, Bm, P, out, send)
     assert ei.value.code == E.ERR_INVALID
     plan.destroy()
+
+
+def test_caller_workspace_first_launch_is_captured_and_allocates_nothing():
+    """With entwine_plan_set_workspace the plan lives in the caller's block: its very first launch
+    can be captured, no launch changes the amount of free device memory, and the results carry the
+    same bits as those of a plan with memory of its own; the layer chain uses the same block."""
+    from paper_2609_11562_b200 import entwine as E
+    wl, rank = WL, 2
+    A, Bm = I.make_operands(wl, device="cuda")
+    P = I.make_peer_partials(wl, device="cuda")
+    res, w = I.make_layer_inputs(wl, device="cuda")
+    out = torch.empty(wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
+    out0, send0 = torch.empty_like(out), torch.empty_like(send)
+    hid, nrm, hid0, nrm0 = (torch.empty_like(out) for _ in range(4))
+    own = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=rank)
+    own.gemm_rs(A, Bm, P, out0, send0)
+    own.last_status()
+    own.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hid0, nrm0, send0)
+    own.last_status()
+    own.destroy()
+
+    plan = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=rank)
+    n = plan.workspace_bytes()
+    assert n >= wl.M * wl.N * 2
+    ws = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(E.EntwineError):
+        plan.set_workspace(ws[1:], n)            # misaligned
+    with pytest.raises(E.EntwineError):
+        plan.set_workspace(ws, n - 256)          # too small
+    plan.set_workspace(ws, n)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            plan.gemm_rs(A, Bm, P, out, send)    # the plan's first launch, inside a capture
+        for _ in range(2):
+            out.fill_(float("nan"))
+            send.fill_(float("nan"))
+            g.replay()
+            side.synchronize()
+            st = plan.last_status()
+            assert st["tiles_reduced"] == plan.counts()["n_reduce"]
+            assert torch.equal(out, out0) and torch.equal(send, send0)
+        plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hid, nrm, send)
+        side.synchronize()
+        plan.last_status()
+        assert torch.equal(hid, hid0) and torch.equal(nrm, nrm0)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    with pytest.raises(E.EntwineError):
+        plan.set_workspace(ws, n)                # after a launch
+    plan.destroy()
+    del g
