@@ -26,7 +26,8 @@
  *
  * Data layout (all bf16, row-major, contiguous)
  *   A             [M, K_local]   rows lda elements apart (ENTWINE_OPT_LDA, default K_local)
- *   B             [N, K_local]   rows ldb elements apart (ENTWINE_OPT_LDB, default K_local): the rank's shard of the layer weight (K contiguous), so the
+ *   B             [N, K_local]   rows ldb elements apart (ENTWINE_OPT_LDB, default K_local): the rank's shard
+ *                                (or [K_local, N] with ENTWINE_OPT_B_LAYOUT = ENTWINE_B_LAYOUT_KN) of the layer weight (K contiguous), so the
  *                                rank's partial output is C = A . B^T, [M, N]
  *   peer_partials [W-1, M, N]    incoming partial outputs of the other ranks in ascending
  *                                rank order (slot q(w) = w < r ? w : w-1).  Only rows
@@ -66,6 +67,9 @@ enum {
   ENTWINE_ERR_INTERNAL  = -5, /* a device-side index check failed                            */
   ENTWINE_ERR_TOO_LARGE = -6  /* the problem does not fit entwine_gemm_rs_static's fixed scratch */
 };
+
+/* Values of ENTWINE_OPT_B_LAYOUT. */
+enum { ENTWINE_B_LAYOUT_NK = 0, ENTWINE_B_LAYOUT_KN = 1 };
 
 /* Values of ENTWINE_OPT_RELEASE_GROUP besides a block count. */
 enum { ENTWINE_RELEASE_PARTITION = -1, ENTWINE_RELEASE_WHOLE = -2 };
@@ -122,6 +126,13 @@ enum {
                                       and >= K_local; 0 (default) = K_local.  May change between
                                       launches                                                     */
   ENTWINE_OPT_LDB             = 17, /* the same for B                                              */
+  ENTWINE_OPT_B_LAYOUT        = 20, /* layout of B.  ENTWINE_B_LAYOUT_NK (default): [N, K_local], K
+                                      contiguous (the shard of an nn.Linear weight); ENTWINE_B_LAYOUT_KN:
+                                      [K_local, N], N contiguous (the C = A . B of Sec. 3.3 as
+                                      written), read by the tensor core as an MN-major operand.  LDB
+                                      is the row pitch of the layout in force; changing the layout
+                                      resets it to contiguous (set LDB after B_LAYOUT).  May change
+                                      between launches                                             */
   ENTWINE_OPT_SPLIT_LAST_WAVE = 19, /* CTA pairs only.  1 (default): when the pair tiles left for the
                                       last wave occupy at most half of the CTA pairs, each of them is
                                       computed as two half-width units (256 x 128: one 128 x 128 tile

@@ -127,6 +127,8 @@ struct KParams {
   int split;      // pair tiles: the last `split` pair tiles of the order are each done as two half-width
                   // units (256 x 128: one 128 x 128 tile per CTA), so that a last wave that fills at
                   // most half of the CTA pairs costs half a tile time; 0 = none
+  int b_kn;       // 1: B is given as [K_local, N] (N contiguous); its stage share is one 3-D TMA box
+                  // [N groups of 64][k rows][64] and the MMA reads it as an MN-major operand
   int kpb;        // k-blocks (64 elements of K) per stage
   int k3d;        // 1: a stage's k-blocks of one operand arrive as ONE 3-D TMA box (the SM's TMA unit keeps
                   // only about two load instructions in flight, so bytes per instruction bound its rate)
@@ -187,6 +189,8 @@ struct KMaps {
   CUtensorMap a, b;      // operands, one k-block per box
   CUtensorMap a3, b3;    // operands viewed as [K/64][rows][64]: one box brings kpb k-blocks (k3d)
   CUtensorMap bh, bh3;   // B with boxes of 64 rows: a CTA's share of a half-width pair tile
+  CUtensorMap bkn, bknh; // B given as [K, N], viewed as [N/64][K][64]: box = kpb*64 k-rows x the CTA's
+                         // groups of 64 columns (whole and half-width units)
   CUtensorMap c_st;      // partial C, box 64 x 128, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
@@ -498,7 +502,21 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   d |= uint64_t(2) << 61;                 // 128-byte swizzle
   return d;
 }
+// The same for an operand stored with its M/N index contiguous ("MN-major": B given as [K, N]):
+// TMA boxes of 64 N-elements (128 bytes, swizzled) x k-rows; 8 k-rows form a 1024-byte swizzle atom,
+// consecutive atoms along K follow each other (stride byte offset 1024), and the next group of 64
+// N-elements lies `group_bytes` further (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t saddr, uint32_t group_bytes) {
+  uint64_t d = 0;
+  d |= uint64_t((saddr & 0x3FFFF) >> 4);
+  d |= uint64_t((group_bytes >> 4) & 0x3FFF) << 16;  // leading byte offset: between 64-element groups of N
+  d |= uint64_t(1024 >> 4) << 32;                    // stride byte offset: between 8-row atoms along K
+  d |= uint64_t(1) << 46;
+  d |= uint64_t(2) << 61;
+  return d;
+}
 // Instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, M = 128.
+// (bit 16 set: B is MN-major)
 template <int BN, int MM>
 __device__ __forceinline__ constexpr uint32_t instr_desc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(MM >> 4) << 24);
@@ -1598,7 +1616,26 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           // k-blocks of this stage that exist (a ragged last stage is filled, and multiplied, in part)
           const int nkb = min(P.kpb, KB - kb0);
           const uint32_t lead_bar = PAIR ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
-          if (P.k3d) {
+          if (P.b_kn) {
+            // B as [K, N]: one box [groups of 64 columns][kpb * 64 k-rows][64], rows past K read as zero;
+            // A as below, k-block by k-block unless its 3-D view exists
+            const uint32_t a_tx = (P.k3d ? P.kpb : nkb) * C::kABytes, b_tx = P.kpb * b_bytes;
+            if (PAIR) {
+              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * (a_tx + b_tx));
+              if (P.k3d) tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
+              else
+                for (int kk = 0; kk < nkb; ++kk)
+                  tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, lead_bar, op_pol);
+              tma_load_3d_pair_hint(b_dst, half < 0 ? &maps.bkn : &maps.bknh, 0, kb0 * kBK, b_row / 64, lead_bar, op_pol);
+            } else {
+              mbar_arrive_expect_tx(full_bar(stage), a_tx + b_tx);
+              if (P.k3d) tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, full_bar(stage), op_pol);
+              else
+                for (int kk = 0; kk < nkb; ++kk)
+                  tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, full_bar(stage), op_pol);
+              tma_load_3d_hint(b_dst, half < 0 ? &maps.bkn : &maps.bknh, 0, kb0 * kBK, b_row / 64, full_bar(stage), op_pol);
+            }
+          } else if (P.k3d) {
             // one box per operand: [kpb k-blocks][rows][64]; k-blocks past the end of K read as zero
             if (PAIR) {
               // both CTAs' bytes are counted on the leader's barrier, which the leader arms
@@ -1637,8 +1674,9 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
-      constexpr uint32_t idesc_full = instr_desc<BN, PAIR ? 256 : 128>();
-      constexpr uint32_t idesc_half = instr_desc<BN / 2, PAIR ? 256 : 128>();
+      const uint32_t b_major_bit = P.b_kn ? (1u << 16) : 0u;
+      const uint32_t idesc_full = instr_desc<BN, PAIR ? 256 : 128>() | b_major_bit;
+      const uint32_t idesc_half = instr_desc<BN / 2, PAIR ? 256 : 128>() | b_major_bit;
       bool ok = true;
 #ifdef ENTWINE_PROFILE
       const long long prof_mma0 = clock64();
@@ -1669,12 +1707,17 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           const int nkb = min(P.kpb, KB - kb0);
           for (int kk = 0; kk < nkb; ++kk) {
             const uint64_t a_desc = smem_desc_sw128(a_s + kk * C::kABytes);
-            const uint64_t b_desc = smem_desc_sw128(b_s + kk * b_bytes);
+            // B K-major: k-block kk of this CTA's rows, K advances by 32 bytes inside a row;
+            // B MN-major: k-rows [64 kk, 64 kk + 64) of every 64-column group (groups kpb * 8 KiB
+            // apart), K advances by 16 rows of 128 bytes
+            const uint64_t b_desc = P.b_kn ? smem_desc_sw128_mn(b_s + kk * (kBK * 128), P.kpb * (kBK * 128))
+                                           : smem_desc_sw128(b_s + kk * b_bytes);
+            const uint32_t b_step = P.b_kn ? (kUmmaK * 128) >> 4 : 2;
 #pragma unroll
             for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // advancing K by 16 elements = 32 bytes = 2 descriptor address units
-              if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb0 | kk | k) != 0);
-              else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb0 | kk | k) != 0);
+              // advancing K by 16 elements = 32 bytes = 2 descriptor address units (K-major)
+              if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + b_step * k, idesc, (kb0 | kk | k) != 0);
+              else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + b_step * k, idesc, (kb0 | kk | k) != 0);
             }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
@@ -2056,17 +2099,33 @@ static bool make_map3(CUtensorMap* map, const void* base, int64_t planes, int64_
 // only where K is a multiple of 64 (the view has no partial k-block).  Returns false on an
 // encoding failure; *k3d tells whether the 3-D maps are usable.
 static bool make_operand_maps(KMaps* maps, const void* A, const void* B, const Geometry& g, int b_rows, int kpb,
-                              int64_t lda, int64_t ldb, int* k3d) {
+                              int64_t lda, int64_t ldb, int b_kn, int* k3d) {
   *k3d = 0;
-  // (bh, bh3: half as many rows of B per box, for the half-width units of a split last wave)
-  if (!make_map(&maps->a, A, g.M, g.K, kBK, kBM, true, lda) || !make_map(&maps->b, B, g.N, g.K, kBK, b_rows, true, ldb) ||
-      !make_map(&maps->bh, B, g.N, g.K, kBK, b_rows / 2, true, ldb))
-    return false;
-  if (kpb < 2 || g.K % kBK != 0) return true;
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  if ((lda > 0 && lda < g.K) || (ldb > 0 && ldb < (b_kn ? g.N : g.K))) return false;
+  // (bh, bh3: half as many rows of B per box, for the half-width units of a split last wave)
+  if (!make_map(&maps->a, A, g.M, g.K, kBK, kBM, true, lda)) return false;
+  if (b_kn) {
+    // B [K, N] seen as [N/64][K][64]: groups of 64 columns are 128 bytes apart inside a row of B
+    for (int h = 0; h < 2; ++h) {
+      const int groups = std::max(1, (h == 0 ? b_rows : b_rows / 2) / 64);
+      cuuint64_t dims[3] = {64, cuuint64_t(g.K), cuuint64_t(g.N / 64)};
+      cuuint64_t strides[2] = {cuuint64_t(ldb > 0 ? ldb : g.N) * 2, 128};
+      cuuint32_t box[3] = {64, cuuint32_t(kBK * kpb), cuuint32_t(groups)};
+      cuuint32_t estr[3] = {1, 1, 1};
+      if (fn(h == 0 ? &maps->bkn : &maps->bknh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(B), dims, strides,
+             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    }
+  } else if (!make_map(&maps->b, B, g.N, g.K, kBK, b_rows, true, ldb) ||
+             !make_map(&maps->bh, B, g.N, g.K, kBK, b_rows / 2, true, ldb)) {
+    return false;
+  }
+  if (kpb < 2 || g.K % kBK != 0) return true;
   bool ok = true;
-  for (int op = 0; op < 3; ++op) {
+  for (int op = 0; op < (b_kn ? 1 : 3); ++op) {
     const int64_t rows = op == 0 ? g.M : g.N;
     const int64_t ld = op == 0 ? (lda > 0 ? lda : g.K) : (ldb > 0 ? ldb : g.K);
     cuuint64_t dims[3] = {cuuint64_t(kBK), cuuint64_t(rows), cuuint64_t(g.K / kBK)};
@@ -2579,7 +2638,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   const void* b_p = (mode != MODE_COMM_ONLY) ? B : d->C;
   const bool comm = mode != MODE_GEMM_ONLY;
   bool ok = (mode != MODE_COMM_ONLY)
-                ? make_operand_maps(&maps, a_p, b_p, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d)
+                ? make_operand_maps(&maps, a_p, b_p, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d)
                 : (make_map(&maps.a, a_p, g.M, g.N, kBK, kBM, true) && make_map(&maps.b, b_p, g.M, g.N, kBK, kBM, true));
   ok = ok && make_map(&maps.c_st, d->C, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
@@ -2724,7 +2783,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   std::memset(&maps, 0, sizeof(maps));
   void* own_buf = own_seg + buf_off;
   const int r = p->rank, W = g.W;
-  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d) &&
+  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d) &&
             make_map(&maps.c_st, own_buf, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, own_buf, g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
@@ -3157,7 +3216,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.split = split_last_wave(p, kp.G);
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
-  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, &kp.k3d) &&
+  bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d) &&
             make_map(&maps.c_st, base, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {

@@ -280,6 +280,11 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);
       return ENTWINE_OK;
+    case ENTWINE_OPT_B_LAYOUT:
+      if (value != ENTWINE_B_LAYOUT_NK && value != ENTWINE_B_LAYOUT_KN) return ENTWINE_ERR_INVALID;
+      if (p->b_kn != (value == ENTWINE_B_LAYOUT_KN ? 1 : 0)) p->ldb = 0;  // the pitch belonged to the other layout
+      p->b_kn = value == ENTWINE_B_LAYOUT_KN ? 1 : 0;
+      return ENTWINE_OK;
     case ENTWINE_OPT_SPLIT_LAST_WAVE:
       if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
       p->split_opt = int(value);
@@ -294,8 +299,11 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       return ENTWINE_OK;
     case ENTWINE_OPT_LDA:
     case ENTWINE_OPT_LDB:
-      // rows start on 16-byte boundaries and do not overlap
-      if (value != 0 && (value < p->g.K || value % 8 != 0 || value > (int64_t(1) << 36))) return ENTWINE_ERR_INVALID;
+      // rows start on 16-byte boundaries (that they do not overlap is checked at the launch, against
+      // the layout in force then)
+      if (value != 0 && (value < 8 || value % 8 != 0 || value > (int64_t(1) << 36))) return ENTWINE_ERR_INVALID;
+      if (value != 0 && key == ENTWINE_OPT_LDA && value < p->g.K) return ENTWINE_ERR_INVALID;
+      if (value != 0 && key == ENTWINE_OPT_LDB && value < (p->b_kn ? p->g.N : p->g.K)) return ENTWINE_ERR_INVALID;
       (key == ENTWINE_OPT_LDA ? p->lda : p->ldb) = value;
       return ENTWINE_OK;
     case ENTWINE_OPT_PREFETCH:

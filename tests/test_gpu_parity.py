@@ -462,3 +462,52 @@ def test_leading_dimensions(wl):
         E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 4, lda=wl.K + 4)      # not a multiple of 8 elements
     with pytest.raises(E.EntwineError):
         E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 4, ldb=wl.K - 8)      # rows would overlap
+
+
+@pytest.mark.parametrize("wl", [SMALL[1], SMALL[2], SMALL[3], SMALL[4]], ids=lambda w: w.name)
+def test_b_given_as_k_by_n(wl):
+    """B as [K_local, N] (ENTWINE_OPT_B_LAYOUT = KN, the C = A . B of Sec. 3.3 as written), contiguous
+    and with a padded row pitch: the fused call against the oracle, and bit for bit against the
+    [N, K_local] call, for CTA pairs and single CTAs, both stage fillings, ragged K, and a plan that
+    switches layouts between launches."""
+    A, Bm = I.make_operands(wl)
+    P = I.make_peer_partials(wl)
+    Ab, Bb, Pb = I.bits(A), I.bits(Bm), I.bits(P)
+    Ad, Bd, Pd = A.cuda(), Bm.cuda(), P.cuda()
+    Bkn = Bd.t().contiguous()                               # [K, N]
+    ldb = wl.N + 24
+    Bkn_pad = torch.full((wl.K, ldb), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Bkn_pad[:, :wl.N] = Bkn
+    r = wl.W - 1
+    BN = 256 if wl.N % 256 == 0 else 128
+    res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, BN, 1, 4)
+    for opts in (dict(), dict(pair_ctas=0), dict(kblocks_per_stage=1), dict(block_n=128)):
+        p0 = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, **opts)
+        out0, send0 = _alloc_outputs(wl)
+        p0.gemm_rs(Ad, Bd, Pd, out0, send0)
+        p0.last_status()
+        p = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, b_layout=E.B_LAYOUT_KN, **opts)
+        out, send = _alloc_outputs(wl)
+        p.gemm_rs(Ad, Bkn, Pd, out, send)
+        st = p.last_status()
+        assert st["tiles_reduced"] == p.counts()["n_reduce"] and st["tiles_pushed"] == p.counts()["n_push"]
+        if _tolerance_is_feasible(wl):
+            _check_against_oracle(wl, r, res, out, send)
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        # padded pitch
+        p.set_option(E.OPT_LDB, ldb)
+        out.fill_(float("nan"))
+        send.fill_(float("nan"))
+        p.gemm_rs(Ad, Bkn_pad, Pd, out, send)
+        p.last_status()
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        # the same plan back on the [N, K] weight (the pitch of the other layout is dropped)
+        p.set_option(E.OPT_B_LAYOUT, E.B_LAYOUT_NK)
+        out.fill_(float("nan"))
+        p.gemm_rs(Ad, Bd, Pd, out, send)
+        p.last_status()
+        assert torch.equal(out, out0) and torch.equal(send, send0)
+        p.destroy()
+        p0.destroy()
+    with pytest.raises(E.EntwineError):
+        E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 4, b_layout=E.B_LAYOUT_KN, ldb=wl.N - 8)
