@@ -126,6 +126,13 @@ enum {
                                       and >= K_local; 0 (default) = K_local.  May change between
                                       launches                                                     */
   ENTWINE_OPT_LDB             = 17, /* the same for B                                              */
+  ENTWINE_OPT_CONSUMER_TMA    = 21, /* 1 (default): once a CTA's producer work is over (and in CTAs
+                                      that do not produce) the consumer streams tiles through a
+                                      shared-memory ring filled by TMA: in pull mode one 3-D box
+                                      whose planes are the peers' heap segments.  0 (needs
+                                      REG_CONSUMER = 1): plain 128-bit loads and stores for the whole
+                                      call, nothing but ordinary loads ever touches peer memory: the
+                                      conservative data path for a first run over NVLink          */
   ENTWINE_OPT_B_LAYOUT        = 20, /* layout of B.  ENTWINE_B_LAYOUT_NK (default): [N, K_local], K
                                       contiguous (the shard of an nn.Linear weight); ENTWINE_B_LAYOUT_KN:
                                       [K_local, N], N contiguous (the C = A . B of Sec. 3.3 as

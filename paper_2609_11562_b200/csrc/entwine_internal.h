@@ -87,6 +87,7 @@ struct Plan {
   int b_kn = 0;             // 1: B is [K_local, N] (N contiguous) instead of [N, K_local]
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int reg_consumer = 1;     // ... from registers (plain loads and stores) instead of a shared-memory TMA ring
+  int consumer_tma = 1;     // 0 (with reg_consumer): the consumer uses plain loads and stores only, to the end
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles
   bool pair = false;        // pair tiles in use for this plan
   int poison = 0;

@@ -141,6 +141,8 @@ struct KParams {
                   // registers (plain loads and stores) instead of a shared-memory ring: ring A then holds
                   // task descriptors only, all shared memory goes to the operand stages, and the SM's TMA
                   // unit serves the operand loads alone
+  int reg_only;   // 1 (with reg_a): the consumer never moves to the TMA ring: every tile, to the end of the
+                  // call and in CTAs that do not produce, goes through registers with plain loads
   int skip_wait;  // treat every flag as published (consumer in isolation)
   int claim;      // most consecutive tasks taken from a list per claim
   int release_group;     // blocks released together (1 = each block by itself; -1, -2: see the header)
@@ -958,6 +960,7 @@ template <bool NORM, bool PULL>
 __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
                                   int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (!NORM && P.reg_a && P.reg_only) start_on_a = true;
   Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P, sh);
 
   if (warp == kCommWarp) {
@@ -970,7 +973,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     const long long MN = (long long)P.M * P.N, RN = P.R * (long long)P.N;
     // moves the pipeline to ring B once the producer's buffers are free
     auto maybe_switch = [&]() {
-      if (ring.id != 0) return;
+      if (ring.id != 0 || (!NORM && P.reg_a && P.reg_only)) return;
       int done = 0;
       if (lane == 0) done = P.early_b ? sh->stages_free : sh->gemm_done;
       done = __shfl_sync(0xffffffffu, done, 0);
@@ -2459,6 +2462,7 @@ static int ring_geometry(const Plan* p, KParams* kp, bool reg_a) {
   // its stages are free
   kp->colocate = (p->colocate && (reg_a || ring_a_bytes >= 2 * kp->slot_bytes[0])) ? 1 : 0;
   kp->reg_a = reg_a ? 1 : 0;
+  kp->reg_only = (reg_a && !p->consumer_tma) ? 1 : 0;
   return ENTWINE_OK;
 }
 

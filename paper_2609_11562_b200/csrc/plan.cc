@@ -280,6 +280,10 @@ int entwine_set_option(entwine_plan_t plan, int key, int64_t value) {
       if (value < 0 || value > 6 || value == 1) return ENTWINE_ERR_INVALID;
       p->stages = int(value);
       return ENTWINE_OK;
+    case ENTWINE_OPT_CONSUMER_TMA:
+      if (value != 0 && value != 1) return ENTWINE_ERR_INVALID;
+      p->consumer_tma = int(value);
+      return ENTWINE_OK;
     case ENTWINE_OPT_B_LAYOUT:
       if (value != ENTWINE_B_LAYOUT_NK && value != ENTWINE_B_LAYOUT_KN) return ENTWINE_ERR_INVALID;
       if (p->b_kn != (value == ENTWINE_B_LAYOUT_KN ? 1 : 0)) p->ldb = 0;  // the pitch belonged to the other layout

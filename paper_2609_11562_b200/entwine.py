@@ -27,6 +27,7 @@ OPT_RANK, OPT_BLOCK_N, OPT_WAIT_BUDGET_NS, OPT_TAIL_HELP = 1, 2, 3, 4
 OPT_WITHHOLD_PEER, OPT_NUM_SMS, OPT_POISON_PARTIAL, OPT_PAIR_CTAS, OPT_COLOCATE = 5, 6, 7, 8, 9
 OPT_PREFETCH, OPT_STAGES, OPT_L2_HINTS, OPT_LISTS, OPT_RELEASE_GROUP = 10, 11, 12, 13, 14
 OPT_KBLOCKS_PER_STAGE, OPT_LDA, OPT_LDB, OPT_REG_CONSUMER, OPT_SPLIT_LAST_WAVE, OPT_B_LAYOUT = 15, 16, 17, 18, 19, 20
+OPT_CONSUMER_TMA = 21
 B_LAYOUT_NK, B_LAYOUT_KN = 0, 1
 RELEASE_PARTITION, RELEASE_WHOLE = -1, -2
 (EXPORT_COUNTS, EXPORT_ORDER, EXPORT_TILES, EXPORT_FLAG_SEQ, EXPORT_LIST_OFFS, EXPORT_TASKS,
@@ -117,7 +118,7 @@ class Plan:
         keys = {"rank": OPT_RANK, "block_n": OPT_BLOCK_N, "wait_budget_ns": OPT_WAIT_BUDGET_NS,
                 "tail_help": OPT_TAIL_HELP, "num_sms": OPT_NUM_SMS, "poison_partial": OPT_POISON_PARTIAL,
                 "pair_ctas": OPT_PAIR_CTAS, "colocate": OPT_COLOCATE, "prefetch": OPT_PREFETCH, "stages": OPT_STAGES, "l2_hints": OPT_L2_HINTS, "lists": OPT_LISTS, "release_group": OPT_RELEASE_GROUP,
-                "kblocks_per_stage": OPT_KBLOCKS_PER_STAGE, "reg_consumer": OPT_REG_CONSUMER, "split_last_wave": OPT_SPLIT_LAST_WAVE, "b_layout": OPT_B_LAYOUT, "lda": OPT_LDA, "ldb": OPT_LDB}
+                "kblocks_per_stage": OPT_KBLOCKS_PER_STAGE, "reg_consumer": OPT_REG_CONSUMER, "split_last_wave": OPT_SPLIT_LAST_WAVE, "b_layout": OPT_B_LAYOUT, "consumer_tma": OPT_CONSUMER_TMA, "lda": OPT_LDA, "ldb": OPT_LDB}
         # num_sms first: it bounds the others
         for name in sorted(options, key=lambda n: {"num_sms": 0, "b_layout": 1}.get(n, 2)):
             self.set_option(keys[name], options[name])

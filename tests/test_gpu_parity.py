@@ -333,6 +333,7 @@ OPTION_SETS = [
     dict(kblocks_per_stage=1), dict(kblocks_per_stage=2, stages=2), dict(kblocks_per_stage=1, stages=6),
     dict(reg_consumer=0), dict(reg_consumer=0, kblocks_per_stage=2, stages=2), dict(reg_consumer=0, kblocks_per_stage=1),
     dict(reg_consumer=0, pair_ctas=0), dict(reg_consumer=1, pair_ctas=0, kblocks_per_stage=1),
+    dict(split_last_wave=0), dict(consumer_tma=0), dict(consumer_tma=0, tail_help=0, colocate=0),
 ]
 
 

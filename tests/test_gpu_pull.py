@@ -45,14 +45,15 @@ class Heap:
         return self.mem[a:a + self.W * Q * 4].view(torch.int32).view(self.W, Q)
 
 
+@pytest.mark.parametrize("consumer_tma", [1, 0], ids=["peer_tiles_by_tma", "peer_tiles_by_plain_loads"])
 @pytest.mark.parametrize("W,M,N,K,order,n_comm", [
     (4, 1024, 768, 192, 1, 0),
     (2, 512, 512, 96, 0, 8),
     (8, 2048, 512, 64, 1, 16),
     (3, 768, 512, 80, 0, 0),
 ])
-def test_every_rank_reduces_its_partition_from_the_heap(W, M, N, K, order, n_comm):
-    plans = [E.Plan(M, N, K, W, order, n_comm, rank=q) for q in range(W)]
+def test_every_rank_reduces_its_partition_from_the_heap(W, M, N, K, order, n_comm, consumer_tma):
+    plans = [E.Plan(M, N, K, W, order, n_comm, rank=q, consumer_tma=consumer_tma) for q in range(W)]
     heap = Heap(plans[0], W, M, N)
     Q = plans[0].counts()["Q"]
     R = M // W

@@ -82,14 +82,14 @@ def test_segment_layout_reported_by_the_planner():
     plan.destroy()
 
 
-def _gpu_worker(rank, world, port, q):
+def _gpu_worker(rank, world, port, q, consumer_tma=1):
     try:
         _init(rank, world, port)
         torch.cuda.set_device(0)  # both ranks on the one GPU
         from oracle import entwine_oracle as O
         from paper_2609_11562_b200 import entwine as E, inputs as I, symheap as SH
         M, N, K = 1024, 512, 128
-        plan = E.Plan(M, N, K, world, 1, 0, rank=rank, wait_budget_ns=50_000_000)
+        plan = E.Plan(M, N, K, world, 1, 0, rank=rank, wait_budget_ns=50_000_000, consumer_tma=consumer_tma)
         seg, flags_off = plan.heap_bytes()
         heap = SH.SymmetricHeap(seg, rank, world, dist, SH.VmmBackend(0))
         Q, R = plan.counts()["Q"], M // world
@@ -133,12 +133,13 @@ def _gpu_worker(rank, world, port, q):
 
 
 @pytest.mark.gpu
-def test_two_processes_share_device_segments_and_reduce_each_others_partials():
+@pytest.mark.parametrize("consumer_tma", [1, 0], ids=["peer_tiles_by_tma", "peer_tiles_by_plain_loads"])
+def test_two_processes_share_device_segments_and_reduce_each_others_partials(consumer_tma):
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 33500 + os.getpid() % 2000
+    port = 33500 + os.getpid() % 2000 + 7 * consumer_tma
     world = 2
-    procs = [ctx.Process(target=_gpu_worker, args=(r, world, port, q)) for r in range(world)]
+    procs = [ctx.Process(target=_gpu_worker, args=(r, world, port, q, consumer_tma)) for r in range(world)]
     for p in procs:
         p.start()
     got = sorted(q.get(timeout=300) for _ in range(world))
