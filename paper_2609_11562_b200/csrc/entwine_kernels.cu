@@ -713,6 +713,10 @@ __device__ __forceinline__ const __nv_bfloat16* peer_base(const KParams& P, int 
   }
   return P.peers + (long long)q * P.M * P.N;
 }
+// ReduceTile of Sec. 4.2 on a whole tile: local contribution first, then the peers in ascending rank
+// order, fp32, one rounding.  A thread's 8 chunks go in batches of 16 / W chunks: all loads of a
+// batch are issued before the first is used.  (A rolling window over the flat sequence of loads was
+// measured too: no faster here, and it spills in the layer-chain kernels.)
 template <int WW, bool PULL>
 __device__ __forceinline__ void reg_reduce_tile(const KParams& P, int ctid, int col, int src_row, int dst_row) {
   constexpr int kChunks = kTile * (kTile * 2 / 16) / kRedThreads;  // 8 per thread
@@ -732,7 +736,6 @@ __device__ __forceinline__ void reg_reduce_tile(const KParams& P, int ctid, int 
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       const int c = ctid + (i0 + b) * kRedThreads;
-      // local contribution first, then the peers in ascending rank order, fp32, one rounding
       float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int q = 0; q < WW; ++q) acc_bf16x8(a, v[b][q]);
@@ -762,6 +765,48 @@ __device__ __forceinline__ void reg_reduce_tile_any(const KParams& P, int ctid, 
         if (q0 + j < P.W - 1) acc_bf16x8(a, v[j]);
     }
     __stcs(reinterpret_cast<uint4*>(P.out + (long long)(dst_row + (c >> 4)) * N + col + (c & 15) * 8), pack_bf16x8(a));
+  }
+}
+// Layer chain (Sec. 5.2.3) from registers: the rank-order fp32 sum, then the residual, one rounding;
+// the bf16 result is the new residual stream (P.out), and the sum of squares of the 128 stored
+// values of each row inside this tile goes to ssq_part (one writer each).  Same arithmetic, in the
+// same order, as the ring path: the sixteen threads of a row add their partial sums by the same
+// shuffles.  WW = 0: any W.
+template <int WW>
+__device__ __forceinline__ void reg_reduce_tile_norm(const KParams& P, int ctid, int lane, int col, int src_row,
+                                                     int dst_row) {
+  constexpr int kChunks = kTile * (kTile * 2 / 16) / kRedThreads;
+  const long long N = P.N;
+#pragma unroll 1
+  for (int i = 0; i < kChunks; ++i) {
+    const int c = ctid + i * kRedThreads;
+    const long long off = (long long)(src_row + (c >> 4)) * N + col + (c & 15) * 8;
+    const long long doff = (long long)(dst_row + (c >> 4)) * N + col + (c & 15) * 8;
+    float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (WW > 0) {
+      uint4 v[WW > 0 ? WW : 1];
+      v[0] = ld_l2_v4(P.cws + off);
+#pragma unroll
+      for (int q = 1; q < WW; ++q) v[q] = ld_stream_v4(peer_base<false>(P, q - 1) + off);
+      const uint4 rv = ld_stream_v4(P.residual + doff);
+#pragma unroll
+      for (int q = 0; q < WW; ++q) acc_bf16x8(a, v[q]);
+      acc_bf16x8(a, rv);
+    } else {
+      acc_bf16x8(a, ld_l2_v4(P.cws + off));
+      for (int q = 1; q < P.W; ++q) acc_bf16x8(a, ld_stream_v4(peer_base<false>(P, q - 1) + off));
+      acc_bf16x8(a, ld_stream_v4(P.residual + doff));
+    }
+    const uint4 o = pack_bf16x8(a);
+    __stcg(reinterpret_cast<uint4*>(P.out + doff), o);  // re-read from L2 by the normalisation
+    float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    acc_bf16x8(h, o);
+    float ssq = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ssq = fmaf(h[e], h[e], ssq);
+#pragma unroll
+    for (int sft = 8; sft > 0; sft >>= 1) ssq += __shfl_xor_sync(0xffffffffu, ssq, sft);
+    if ((lane & 15) == 0) __stcg(&P.ssq_part[(long long)(dst_row + (c >> 4)) * P.nTn + col / kTile], ssq);
   }
 }
 __device__ __forceinline__ void reg_push_tile(const KParams& P, int ctid, int col, int src_row, int dst_row) {
@@ -825,10 +870,15 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
       else if (P.W == 8) reg_reduce_tile<8, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       else reg_reduce_tile_any<PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       if (ctid == 0) PROF_ADD(10);
-    } else if (!NORM && !PULL && m.kind == 5) {
+    } else if (!PULL && m.kind == 5) {
       PROF_T0();
       reg_push_tile(P, ctid, m.dst_x, m.aux, m.dst_y);
       if (ctid == 0) PROF_ADD(11);
+    } else if (NORM && !PULL && m.kind == 4) {
+      if (P.W == 2) reg_reduce_tile_norm<2>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
+      else if (P.W == 4) reg_reduce_tile_norm<4>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
+      else if (P.W == 8) reg_reduce_tile_norm<8>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
+      else reg_reduce_tile_norm<0>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
     } else if (!NORM && m.kind == 0) {
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
       const int rs = ring.rs, sub_bytes = ring.sub_bytes;
@@ -1199,7 +1249,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           }
           maybe_switch();
           if (!ok) break;
-          if (!NORM && ring.id == 0 && P.reg_a) {
+          if (ring.id == 0 && P.reg_a) {
             // register path: the reducing warps load the tile themselves; one descriptor per task
             bool slot_ok = true;
             if (lane == 0) {
@@ -1350,6 +1400,28 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         }
         i = __shfl_sync(0xffffffffu, i, 0);
         if (i >= P.Q) break;
+        if (ring.id == 0 && P.reg_a) {
+          // the descriptor ring has no memory for the rows to normalise: wait (boundedly) until the
+          // CTA's operand stages are free, then move to ring B
+          bool open = true;
+          if (lane == 0) {
+            unsigned long long t0 = 0;
+            for (uint32_t spins = 1; !(P.early_b ? sh->stages_free : sh->gemm_done); ++spins) {
+              __nanosleep(128);
+              if ((spins % kSpinCheck) == 0) {
+                if (sh->abort) { open = false; break; }
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > 64ULL * P.wait_budget_ns) { open = false; break; }
+              }
+            }
+          }
+          ok = __all_sync(0xffffffffu, open);
+          if (!ok) {
+            if (lane == 0) report(P, -ENTWINE_ERR_TIMEOUT, -7);
+            break;
+          }
+        }
         maybe_switch();
         if (!ok) break;
         issue_norm_run(i, kRun);
@@ -1411,10 +1483,11 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         break;
       }
       if (m.kind == 0 || m.kind >= 4 || (NORM && (m.kind == 2 || m.kind == 3))) {
-        if (NORM && m.kind == 0 && m.aux >= 0) {
-          // layer chain: the last step of a reduce task counts its tile in the band
+        if (NORM && ((m.kind == 0 && m.aux >= 0) || m.kind == 4)) {
+          // layer chain: the last step of a reduce task (or a whole task done from registers,
+          // whose first destination row is dst_y) counts its tile in the band
           fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
-          atomicAdd(&P.band_ctr[m.aux], 1u);
+          atomicAdd(&P.band_ctr[m.kind == 4 ? m.dst_y / kTile : m.aux], 1u);
         }
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
@@ -2592,7 +2665,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  rc = ring_geometry(p, &kp, p->reg_consumer && !norm);
+  rc = ring_geometry(p, &kp, p->reg_consumer != 0);
   if (rc != ENTWINE_OK) return rc;
   kp.prefetch = p->prefetch;
   kp.l2_hints = p->l2_hints;
