@@ -3,7 +3,7 @@ Sec. 4.3: the communication budget, the tile order and the producer's configurat
 together, by end-to-end latency, once per shape).
 
 For one shape (M, N, K_local, W) the tuner times the fused call over a grid of
-(tile order, n_comm_sms, operand stages, block width BN), keeps the fastest and reports next to
+(tile order, n_comm_sms, producer configuration, block width BN), keeps the fastest and reports next to
 it the quantities of the paper's budget model: the communication volume of Eq. 2 (here with the
 push traffic of the one-GPU emulation), the computation window T_G of Eq. 3 as measured with the
 chosen budget, and the bandwidth B_req = V / T_G that the consumer side must sustain to finish
@@ -21,9 +21,18 @@ import os
 import statistics
 
 ORDERS = {"row_major": 0, "interleaved": 1}
-DEFAULT = {"tile_order": "interleaved", "n_comm_sms": 0, "stages": 0, "block_n": 256}
+DEFAULT = {"tile_order": "interleaved", "n_comm_sms": 0, "stages": 0, "block_n": 256, "kblocks_per_stage": 0,
+           "reg_consumer": 1}
 BUDGETS = (0, 8, 16, 32)
-STAGES = (0, 3, 4, 5)
+# Producer / co-located-consumer configurations tried per (order, budget): operand-ring stages
+# (0 = automatic), k-blocks per stage (0 = automatic: two where a stage then is two 32 KiB boxes) and
+# whether the consumer warps of a producing CTA move tiles through registers or through a TMA ring.
+PRODUCER = ({"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 1},
+            {"stages": 2, "kblocks_per_stage": 0, "reg_consumer": 1},
+            {"stages": 0, "kblocks_per_stage": 1, "reg_consumer": 1},
+            {"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 0},
+            {"stages": 0, "kblocks_per_stage": 1, "reg_consumer": 0})
+STAGES = (0, 3, 4, 5)  # (kept for callers that pass a stage list of their own)
 TIE = 1.03  # a configuration must beat the default by more than this factor to replace it:
             # repeated measurements of one configuration differ by 1-2 % (event timer, clocks)
 
@@ -57,12 +66,21 @@ def launch_options(table, M, N, K_local, W):
     cfg = dict(DEFAULT)
     if table:
         cfg.update(table.get("shapes", {}).get(shape_key(M, N, K_local, W), {}).get("best", {}))
+    return ORDERS[cfg["tile_order"]], int(cfg["n_comm_sms"]), _plan_options(cfg)
+
+
+def _plan_options(cfg):
+    """The plan options of a configuration: whatever differs from the library's defaults."""
     opts = {}
-    if cfg["stages"]:
+    if cfg.get("stages", 0):
         opts["stages"] = int(cfg["stages"])
-    if cfg["block_n"] != 256:
+    if cfg.get("block_n", 256) != 256:
         opts["block_n"] = int(cfg["block_n"])
-    return ORDERS[cfg["tile_order"]], int(cfg["n_comm_sms"]), opts
+    if cfg.get("kblocks_per_stage", 0):
+        opts["kblocks_per_stage"] = int(cfg["kblocks_per_stage"])
+    if cfg.get("reg_consumer", 1) != 1:
+        opts["reg_consumer"] = int(cfg["reg_consumer"])
+    return opts
 
 
 def load_table(path):
@@ -96,7 +114,7 @@ def _time(fn, flush, torch, iters, warmup=2):
     return statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
 
 
-def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=STAGES, ranks=None):
+def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=None, ranks=None, producer=PRODUCER):
     """Times the grid on the current CUDA device and returns the table entry of the shape.
 
     A configuration's latency is the largest over the emulated ranks tried (first, middle, last
@@ -112,12 +130,12 @@ def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=STAGES, ranks=None):
     send = torch.empty(wl.W - 1, wl.R, wl.N, dtype=torch.bfloat16, device="cuda")
     points = []
 
-    def measure(order_name, n_comm, stg, bn):
-        opts = {}
-        if stg:
-            opts["stages"] = stg
-        if bn != 256:
-            opts["block_n"] = bn
+    if stages is not None:  # a plain list of stage counts, the other producer settings at their defaults
+        producer = tuple({"stages": s, "kblocks_per_stage": 0, "reg_consumer": 1} for s in stages)
+
+    def measure(order_name, n_comm, prod, bn):
+        cfg = dict(prod, block_n=bn)
+        opts = _plan_options(cfg)
         worst = None
         for rank in ranks:
             try:
@@ -132,22 +150,24 @@ def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=STAGES, ranks=None):
                 return None
             plan.destroy()
             if worst is None or us > worst["fused_us"]:
-                worst = {"tile_order": order_name, "n_comm_sms": n_comm, "stages": stg, "block_n": bn,
-                         "fused_us": us, "slowest_rank": rank, "t_gemm_us": st["t_gemm_ns"] / 1e3,
-                         "t_end_us": st["t_end_ns"] / 1e3}
+                worst = dict(cfg, tile_order=order_name, n_comm_sms=n_comm,
+                             fused_us=us, slowest_rank=rank, t_gemm_us=st["t_gemm_ns"] / 1e3,
+                             t_end_us=st["t_end_ns"] / 1e3)
         points.append(worst)
         return worst
 
     for order_name in ORDERS:
         for n_comm in budgets:
-            for stg in stages:
-                measure(order_name, n_comm, stg, 256)
+            for prod in producer:
+                measure(order_name, n_comm, prod, 256)
+    points[:] = [r for r in points if r is not None]
     best = min(points, key=lambda r: r["fused_us"])
     if wl.N % 128 == 0:
         # the narrow producer block with the winner's other settings
-        measure(best["tile_order"], best["n_comm_sms"], best["stages"], 128)
+        measure(best["tile_order"], best["n_comm_sms"], {k: best[k] for k in producer[0]}, 128)
+        points[:] = [r for r in points if r is not None]
         best = min(points, key=lambda r: r["fused_us"])
-    default = next(r for r in points if all(r[k] == DEFAULT[k] for k in DEFAULT))
+    default = next(r for r in points if all(r.get(k, DEFAULT[k]) == DEFAULT[k] for k in DEFAULT))
     if default["fused_us"] <= TIE * best["fused_us"]:
         best = default  # within measurement noise of the default: keep the default
     t_g = best["t_gemm_us"] * 1e-6

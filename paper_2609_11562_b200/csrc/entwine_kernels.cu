@@ -88,10 +88,9 @@ constexpr int kRegSlots = 4;       // task descriptors in flight between the cla
 constexpr int kMaxStages = 6;
 constexpr int kBarOff = kDataBytes;
 constexpr int kBarBytes = 640;
-constexpr int kBarGemm = 0;        // full[6], empty[6], tfull[2], tempty[2]
+constexpr int kBarGemm = 0;        // full[6], empty[6], tfull[2], tempty[2]; 152..191 unused
 constexpr int kBarTmemSlot = 136;
 constexpr int kBarPair = 144;      // end-of-producer handshake of a CTA pair
-constexpr int kBarStaging = 152;   // staged[2], free[2]: epilogue warps <-> publishing warp
 constexpr int kBarRingA = 192;     // full[8], empty[8], reduced[8]
 constexpr int kBarRingB = 192 + 192;
 constexpr int kSmemBytes = kBarOff + kBarBytes + 1024;  // + alignment slack
@@ -193,7 +192,6 @@ struct KMaps {
   CUtensorMap bh, bh3;   // B with boxes of 64 rows: a CTA's share of a half-width pair tile
   CUtensorMap bkn, bknh; // B given as [K, N], viewed as [N/64][K][64]: box = kpb*64 k-rows x the CTA's
                          // groups of 64 columns (whole and half-width units)
-  CUtensorMap c_st;      // partial C, box 64 x 128, swizzled (epilogue stores)
   // consumer maps, one set per ring (the box height is the ring's rs)
   CUtensorMap c_ld[2];      // partial C, box 128 x rs: the local rows of a reduce step
   CUtensorMap p_ld[2];      // incoming partials as a 3-D tensor [W-1][M][N], box 128 x rs x (W-1):
@@ -282,11 +280,6 @@ __device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, int x,
                                                   uint64_t policy) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
                ::"l"(map), "r"(x), "r"(y), "r"(src), "l"(policy)
-               : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(map), "r"(x), "r"(y), "r"(src)
                : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int x, int y) {
@@ -432,9 +425,6 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-__device__ __forceinline__ void st_release_cta(int* p, int v) {
-  asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ void red_release_cta_add(int* p, int v) {
   asm volatile("red.release.cta.shared::cta.add.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
@@ -1556,8 +1546,6 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   const int stage_bytes = P.kpb * C::kKBlockBytes;
   const uint32_t tmem_slot = smem_base + kBarOff + kBarTmemSlot;
   const uint32_t pair_bar = smem_base + kBarOff + kBarPair;
-  auto staged_bar = [&](int b) { return smem_base + kBarOff + kBarStaging + 8u * b; };
-  auto sfree_bar = [&](int b) { return smem_base + kBarOff + kBarStaging + 8u * (2 + b); };
   const bool is_producer = (int)blockIdx.x < P.G && P.mode != MODE_COMM_ONLY;
   const int g = (int)blockIdx.x;                 // producer index
   const int cidx = (int)blockIdx.x - P.G;        // consumer index of a dedicated consumer CTA
@@ -1613,10 +1601,6 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         mbar_init(tempty_bar(a), (PAIR ? 2 : 1) * (kEpiThreads / 32));
       }
       mbar_init(pair_bar, 1);
-      for (int b = 0; b < 2; ++b) {
-        mbar_init(staged_bar(b), kEpiThreads / 32);
-        mbar_init(sfree_bar(b), 1);
-      }
     }
     for (int ring = 0; ring < 2; ++ring) {  // consumer rings: full, empty, reduced
       const uint32_t rb = smem_base + kBarOff + (ring == 0 ? kBarRingA : kBarRingB);
@@ -2717,8 +2701,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   bool ok = (mode != MODE_COMM_ONLY)
                 ? make_operand_maps(&maps, a_p, b_p, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d)
                 : (make_map(&maps.a, a_p, g.M, g.N, kBK, kBM, true) && make_map(&maps.b, b_p, g.M, g.N, kBK, kBM, true));
-  ok = ok && make_map(&maps.c_st, d->C, g.M, g.N, 64, kBM, true) &&
-            make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
+  ok = ok && make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
     const int prs = kp.prs[id];
@@ -2861,7 +2844,6 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   void* own_buf = own_seg + buf_off;
   const int r = p->rank, W = g.W;
   bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d) &&
-            make_map(&maps.c_st, own_buf, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, own_buf, g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
@@ -3294,7 +3276,6 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   KMaps maps;
   std::memset(&maps, 0, sizeof(maps));
   bool ok = make_operand_maps(&maps, A, B, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d) &&
-            make_map(&maps.c_st, base, g.M, g.N, 64, kBM, true) &&
             make_map(&maps.p_pf, peer_partials, int64_t(g.W - 1) * g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];

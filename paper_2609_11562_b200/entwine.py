@@ -231,8 +231,7 @@ class Plan:
     def last_sm_clock_mhz(self) -> float:
         """SM clock of the launch that the last last_status() call reported (0.0 if unknown)."""
         out = (_i64 * 2)()
-        _check(_lib.entwine_last_sm_clock(self._h, out), "entwine_last_sm_clock",
-           "entwine_plan_workspace_bytes", "entwine_plan_set_workspace")
+        _check(_lib.entwine_last_sm_clock(self._h, out), "entwine_last_sm_clock")
         return out[0] / out[1] * 1e3 if out[1] > 0 else 0.0
 
     def destroy(self):
