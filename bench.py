@@ -520,21 +520,21 @@ def run_layer_chain(args, peaks, flush, torch, E, I):
             plan.comm_only(Cfull, P, out, send, 0)
             return rest()
 
-        one_reg = med(time_steps(lambda: plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send),
+        one_ring = med(time_steps(lambda: plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send),
                                  iters, 3, flush, torch))
         st = plan.last_status()
-        # the same launch with the co-located consumer on the shared-memory TMA ring instead of
-        # registers (plan option reg_consumer = 0): which of the two is faster depends on the shape
-        # (few, long reduce tasks per CTA favour the ring), so both are timed and the faster is the
-        # chain's figure, as the tuner does for the plain call
-        ring_plan = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=wl.W - 1, reg_consumer=0)
-        one_ring = med(time_steps(lambda: ring_plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send),
+        # the same launch with the co-located consumer moving whole tiles through registers instead
+        # of the shared-memory TMA ring (plan option reg_consumer = 1): which of the two is faster
+        # depends on the shape (few, long reduce tasks per CTA favour the ring), so both are timed and
+        # the faster is the chain's figure, as the tuner does for the plain call
+        reg_plan = E.Plan(wl.M, wl.N, wl.K, wl.W, 1, 0, rank=wl.W - 1, reg_consumer=1)
+        one_reg = med(time_steps(lambda: reg_plan.gemm_rs_norm(A, Bm, P, res, w, 1e-5, hidden, normed, send),
                                   iters, 3, flush, torch))
-        st_ring = ring_plan.last_status()
-        ring_plan.destroy()
+        st_reg = reg_plan.last_status()
+        reg_plan.destroy()
         one = min(one_reg, one_ring)
-        if one_ring < one_reg:
-            st = st_ring
+        if one_reg < one_ring:
+            st = st_reg
         two = med(time_steps(fused_then_library, iters, 3, flush, torch))
         plan.last_status()
         three = med(time_steps(unfused, iters, 3, flush, torch))
@@ -549,7 +549,7 @@ def run_layer_chain(args, peaks, flush, torch, E, I):
         plan.destroy()
         report[f"seq_{seq}"] = {
             "shape": {"W": wl.W, "M": wl.M, "N": wl.N, "K_local": wl.K},
-            "one_launch_us": one, "one_launch_consumer": "registers" if one_reg <= one_ring else "tma_ring",
+            "one_launch_us": one, "one_launch_consumer": "registers" if one_reg < one_ring else "tma_ring",
             "one_launch_registers_us": one_reg, "one_launch_tma_ring_us": one_ring,
             "gemm_rs_then_library_add_norm_us": two,
             "cublas_reduce_add_norm_us": three, "gemm_rs_alone_us": rs_only,

@@ -129,10 +129,11 @@ enum {
   ENTWINE_OPT_CONSUMER_TMA    = 21, /* 1 (default): once a CTA's producer work is over (and in CTAs
                                       that do not produce) the consumer streams tiles through a
                                       shared-memory ring filled by TMA: in pull mode one 3-D box
-                                      whose planes are the peers' heap segments.  0 (needs
-                                      REG_CONSUMER = 1): plain 128-bit loads and stores for the whole
-                                      call, nothing but ordinary loads ever touches peer memory: the
-                                      conservative data path for a first run over NVLink          */
+                                      whose planes are the peers' heap segments.  0 (implies the
+                                      register path of REG_CONSUMER): plain 128-bit loads and stores
+                                      for the whole call, nothing but ordinary loads ever touches
+                                      peer memory: the conservative data path for a first run over
+                                      NVLink                                                       */
   ENTWINE_OPT_B_LAYOUT        = 20, /* layout of B.  ENTWINE_B_LAYOUT_NK (default): [N, K_local], K
                                       contiguous (the shard of an nn.Linear weight); ENTWINE_B_LAYOUT_KN:
                                       [K_local, N], N contiguous (the C = A . B of Sec. 3.3 as
@@ -148,13 +149,15 @@ enum {
                                       be any multiple of the reduction tile, Sec. 4.2); 0: whole
                                       pair tiles only.  Off with a release group other than 1      */
   ENTWINE_OPT_REG_CONSUMER    = 18, /* how the consumer warps of a CTA that still produces move their
-                                      tiles.  1 (default): whole tiles through registers with plain
-                                      128-bit loads and stores, so that all shared memory and the
-                                      SM's TMA unit serve the operand ring; 0: through a small
-                                      shared-memory ring filled by TMA beside the operand stages.
+                                      tiles.  0 (default): through a small shared-memory ring filled
+                                      by TMA beside the operand stages; 1: whole tiles through
+                                      registers with plain 128-bit loads and stores, so that all
+                                      shared memory and the SM's TMA unit serve the operand ring
+                                      (measured slower on the benchmark's shapes: the loads of eight
+                                      warps stretch the producer more than the ring does; a kernel
+                                      of its own, so that neither path's code weighs on the other).
                                       Once a CTA's producer work is over (and in dedicated consumer
-                                      CTAs) tiles always go through the large TMA ring.  The layer
-                                      chain always uses the ring                                   */
+                                      CTAs) tiles go through the large TMA ring either way          */
   ENTWINE_OPT_COLOCATE        = 9  /* 1 (default): with TAIL_HELP (or n_comm_sms = 0) a producer
                                       CTA's consumer warps take tasks while its tensor-core work
                                       is still running, through a small shared-memory ring beside

@@ -22,16 +22,17 @@ import statistics
 
 ORDERS = {"row_major": 0, "interleaved": 1}
 DEFAULT = {"tile_order": "interleaved", "n_comm_sms": 0, "stages": 0, "block_n": 256, "kblocks_per_stage": 0,
-           "reg_consumer": 1}
+           "reg_consumer": 0}
 BUDGETS = (0, 8, 16, 32)
 # Producer / co-located-consumer configurations tried per (order, budget): operand-ring stages
-# (0 = automatic), k-blocks per stage (0 = automatic: two where a stage then is two 32 KiB boxes) and
-# whether the consumer warps of a producing CTA move tiles through registers or through a TMA ring.
-PRODUCER = ({"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 1},
-            {"stages": 2, "kblocks_per_stage": 0, "reg_consumer": 1},
-            {"stages": 0, "kblocks_per_stage": 1, "reg_consumer": 1},
-            {"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 0},
-            {"stages": 0, "kblocks_per_stage": 1, "reg_consumer": 0})
+# (0 = automatic), k-blocks per stage (0 = automatic: one beside a consumer ring, two with the register
+# consumer where a stage then is two 32 KiB boxes) and whether the consumer warps of a producing CTA
+# move tiles through a TMA ring or through registers.
+PRODUCER = ({"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 0},
+            {"stages": 4, "kblocks_per_stage": 0, "reg_consumer": 0},
+            {"stages": 3, "kblocks_per_stage": 0, "reg_consumer": 0},
+            {"stages": 0, "kblocks_per_stage": 0, "reg_consumer": 1},
+            {"stages": 0, "kblocks_per_stage": 1, "reg_consumer": 1})
 STAGES = (0, 3, 4, 5)  # (kept for callers that pass a stage list of their own)
 TIE = 1.03  # a configuration must beat the default by more than this factor to replace it:
             # repeated measurements of one configuration differ by 1-2 % (event timer, clocks)
@@ -78,7 +79,7 @@ def _plan_options(cfg):
         opts["block_n"] = int(cfg["block_n"])
     if cfg.get("kblocks_per_stage", 0):
         opts["kblocks_per_stage"] = int(cfg["kblocks_per_stage"])
-    if cfg.get("reg_consumer", 1) != 1:
+    if cfg.get("reg_consumer", 0) != 0:
         opts["reg_consumer"] = int(cfg["reg_consumer"])
     return opts
 
@@ -131,7 +132,7 @@ def tune_shape(wl, flush, iters=8, budgets=BUDGETS, stages=None, ranks=None, pro
     points = []
 
     if stages is not None:  # a plain list of stage counts, the other producer settings at their defaults
-        producer = tuple({"stages": s, "kblocks_per_stage": 0, "reg_consumer": 1} for s in stages)
+        producer = tuple({"stages": s, "kblocks_per_stage": 0, "reg_consumer": 0} for s in stages)
 
     def measure(order_name, n_comm, prod, bn):
         cfg = dict(prod, block_n=bn)

@@ -86,8 +86,8 @@ struct Plan {
   int64_t lda = 0, ldb = 0; // leading dimensions of A and B in elements, 0 = contiguous
   int b_kn = 0;             // 1: B is [K_local, N] (N contiguous) instead of [N, K_local]
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
-  int reg_consumer = 1;     // ... from registers (plain loads and stores) instead of a shared-memory TMA ring
-  int consumer_tma = 1;     // 0 (with reg_consumer): the consumer uses plain loads and stores only, to the end
+  int reg_consumer = 0;     // 1: ... from registers (plain loads and stores) instead of a shared-memory TMA ring
+  int consumer_tma = 1;     // 0: the consumer uses plain loads and stores only, to the end (implies the register path)
   int pair_opt = 1;         // allow CTA-pair (256 x 256) producer tiles
   bool pair = false;        // pair tiles in use for this plan
   int poison = 0;

@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 
 #include "entwine_internal.h"
 
@@ -661,6 +662,7 @@ struct Ring {
   __device__ __forceinline__ uint32_t empty(int s) const { return bars + 8u * (kMaxSlots + s); }
   __device__ __forceinline__ uint32_t red(int s) const { return bars + 8u * (2 * kMaxSlots + s); }
 };
+template <bool REG>
 __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KParams& P, const CtaShared* sh) {
   Ring r;
   r.id = id;
@@ -672,7 +674,7 @@ __device__ __forceinline__ Ring make_ring(uint32_t smem_base, int id, const KPar
   r.slot_bytes = P.slot_bytes[r.geom];
   r.sub_bytes = r.rs * kTile * 2;
   r.n_slots = min(kMaxSlots, (id == 0 ? P.ring_a_bytes : sh->ring_b_bytes) / r.slot_bytes);
-  if (id == 0 && P.reg_a) r.n_slots = kRegSlots;  // descriptors only
+  if (REG && id == 0) r.n_slots = kRegSlots;  // descriptors only
   return r;
 }
 
@@ -818,7 +820,7 @@ __device__ __forceinline__ void reg_push_tile(const KParams& P, int ctid, int co
 // The reducing warps' loop (Sec. 4.2, ReduceTile).  NORM selects the layer-chain variant, which
 // carries the tile's residual in registers and handles the residual and normalisation steps; the
 // plain variant is compiled without any of that state.
-template <bool NORM, bool PULL>
+template <bool NORM, bool PULL, bool REG>
 __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, uint32_t smem_base, Ring ring) {
   const int lane = threadIdx.x & 31;
   const int ctid = threadIdx.x - kRedWarp0 * 32;
@@ -847,12 +849,12 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
     const SlotMeta m = sh->meta[ring.id][slot];
     if (m.kind == -1) break;
     if (m.kind == -2) {
-      ring = make_ring(smem_base, 1, P, sh);
+      ring = make_ring<REG>(smem_base, 1, P, sh);
       slot = -1;
       ph = 0;
       continue;
     }
-    if (!NORM && m.kind == 4) {
+    if (REG && !NORM && m.kind == 4) {
       // a whole reduce task from registers (ReduceTile of Sec. 4.2 on all 128 rows of the tile)
       PROF_T0();
       if (P.W == 2) reg_reduce_tile<2, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
@@ -860,11 +862,11 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
       else if (P.W == 8) reg_reduce_tile<8, PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       else reg_reduce_tile_any<PULL>(P, ctid, m.dst_x, m.aux, m.dst_y);
       if (ctid == 0) PROF_ADD(10);
-    } else if (!PULL && m.kind == 5) {
+    } else if (REG && !PULL && m.kind == 5) {
       PROF_T0();
       reg_push_tile(P, ctid, m.dst_x, m.aux, m.dst_y);
       if (ctid == 0) PROF_ADD(11);
-    } else if (NORM && !PULL && m.kind == 4) {
+    } else if (REG && NORM && !PULL && m.kind == 4) {
       if (P.W == 2) reg_reduce_tile_norm<2>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
       else if (P.W == 4) reg_reduce_tile_norm<4>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
       else if (P.W == 8) reg_reduce_tile_norm<8>(P, ctid, lane, m.dst_x, m.aux, m.dst_y);
@@ -996,12 +998,12 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
 // and write the result; warp 3 forwards pushed tiles with TMA stores and recycles the slots.
 // In a producer CTA the pipeline starts on the small ring A beside the producer's buffers and
 // moves to ring B (the producer's buffers) once `gemm_done` is set.
-template <bool NORM, bool PULL>
+template <bool NORM, bool PULL, bool REG>
 __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps& maps, CtaShared* sh, uint32_t smem_base,
                                   int first_list, int n_lists, bool start_on_a, CommCounters* cnt) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (!NORM && P.reg_a && P.reg_only) start_on_a = true;
-  Ring ring = make_ring(smem_base, start_on_a ? 0 : 1, P, sh);
+  if (REG && !NORM && P.reg_only) start_on_a = true;
+  Ring ring = make_ring<REG>(smem_base, start_on_a ? 0 : 1, P, sh);
 
   if (warp == kCommWarp) {
     // ---------------- claim, poll, load ----------------
@@ -1013,7 +1015,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     const long long MN = (long long)P.M * P.N, RN = P.R * (long long)P.N;
     // moves the pipeline to ring B once the producer's buffers are free
     auto maybe_switch = [&]() {
-      if (ring.id != 0 || (!NORM && P.reg_a && P.reg_only)) return;
+      if (ring.id != 0 || (REG && !NORM && P.reg_only)) return;
       int done = 0;
       if (lane == 0) done = P.early_b ? sh->stages_free : sh->gemm_done;
       done = __shfl_sync(0xffffffffu, done, 0);
@@ -1026,7 +1028,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         // must have returned its slot first: slot s has been used uses(s) times; its last use,
         // number uses(s) - 1, is over when its empty barrier completes the phase of that parity.
         // (In register mode ring A holds no data at all.)
-        for (int sl = 0; !P.early_b && !P.reg_a && free_slot && sl < ring.n_slots; ++sl) {
+        for (int sl = 0; !P.early_b && !REG && free_slot && sl < ring.n_slots; ++sl) {
           const int uses = (it - sl + ring.n_slots - 1) / ring.n_slots;
           if (uses > 0) free_slot = mbar_wait(ring.empty(sl), (uses - 1) & 1, P, sh);
         }
@@ -1039,7 +1041,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         }
       }
       ok = __all_sync(0xffffffffu, free_slot);
-      ring = make_ring(smem_base, 1, P, sh);
+      ring = make_ring<REG>(smem_base, 1, P, sh);
       it = 0;
     };
     // Layer chain: normalisation tasks (one per tile of the rank's partition, band by band) are
@@ -1239,7 +1241,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
           }
           maybe_switch();
           if (!ok) break;
-          if (ring.id == 0 && P.reg_a) {
+          if (REG && ring.id == 0) {
             // register path: the reducing warps load the tile themselves; one descriptor per task
             bool slot_ok = true;
             if (lane == 0) {
@@ -1390,7 +1392,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         }
         i = __shfl_sync(0xffffffffu, i, 0);
         if (i >= P.Q) break;
-        if (ring.id == 0 && P.reg_a) {
+        if (REG && ring.id == 0) {
           // the descriptor ring has no memory for the rows to normalise: wait (boundedly) until the
           // CTA's operand stages are free, then move to ring B
           bool open = true;
@@ -1429,7 +1431,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     __syncwarp();
   } else if (warp >= kRedWarp0 && warp < kRedWarp0 + kRedThreads / 32) {
     // ---------------- ReduceTile on the slots (Sec. 4.2) ----------------
-    reducer_role<NORM, PULL>(P, sh, smem_base, ring);
+    reducer_role<NORM, PULL, REG>(P, sh, smem_base, ring);
   } else if (warp == kStoreWarp && lane == 0) {
     // ---------------- forward push slots with TMA stores, recycle all slots ----------------
     // Push stores are kept in flight: a pushed slot is released once its store has read it,
@@ -1443,7 +1445,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       if (!n_pend) return;
       bulk_wait_read<0>();
       for (; n_pend > 0; --n_pend, pend >>= 8) {
-        const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P, sh);
+        const Ring rr = make_ring<REG>(smem_base, int(pend >> 4) & 1, P, sh);
         mbar_arrive(rr.empty(int(pend & 15u)));
       }
     };
@@ -1462,7 +1464,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
       if (m.kind == -1) break;
       if (m.kind == -2) {
         retire_all();
-        ring = make_ring(smem_base, 1, P, sh);
+        ring = make_ring<REG>(smem_base, 1, P, sh);
         slot = -1;
         ph = 0;
         continue;
@@ -1472,12 +1474,12 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         sh->abort = 1;
         break;
       }
-      if (m.kind == 0 || m.kind >= 4 || (NORM && (m.kind == 2 || m.kind == 3))) {
-        if (NORM && ((m.kind == 0 && m.aux >= 0) || m.kind == 4)) {
+      if (m.kind == 0 || (REG && m.kind >= 4) || (NORM && (m.kind == 2 || m.kind == 3))) {
+        if (NORM && ((m.kind == 0 && m.aux >= 0) || (REG && m.kind == 4))) {
           // layer chain: the last step of a reduce task (or a whole task done from registers,
           // whose first destination row is dst_y) counts its tile in the band
           fence_acq_rel_gpu();  // the reducing warps' stores (seen through the barrier) first
-          atomicAdd(&P.band_ctr[m.kind == 4 ? m.dst_y / kTile : m.aux], 1u);
+          atomicAdd(&P.band_ctr[(REG && m.kind == 4) ? m.dst_y / kTile : m.aux], 1u);
         }
         mbar_arrive(ring.empty(slot));  // reduced and written out by the reducing warps
       } else {
@@ -1485,7 +1487,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
-          const Ring rr = make_ring(smem_base, int(pend >> 4) & 1, P, sh);
+          const Ring rr = make_ring<REG>(smem_base, int(pend >> 4) & 1, P, sh);
           mbar_arrive(rr.empty(int(pend & 15u)));
           pend >>= 8;
           --n_pend;
@@ -1526,7 +1528,7 @@ entwine_reset_kernel(unsigned* flags, int n_flags, int* heads, int n_heads, Stat
 // ------------------------------------------------------------------------------------------
 // NORM: the layer-chain variant (residual add + RMSNorm in the consumer) is a kernel of its own,
 // so that the plain kernel's code and register allocation are untouched by it.
-template <int BN, bool PAIR, bool NORM, bool PULL>
+template <int BN, bool PAIR, bool NORM, bool PULL, bool REG>
 __global__ void __launch_bounds__(kThreads, 1)
 entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
   using C = Cfg<BN, PAIR>;
@@ -1647,14 +1649,18 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       return p;
     };
 
-    if (warp == kTmaWarp && lane == 0) {
-      // ---- TMA producer (every CTA loads its own operands) ----
+    // The two single-thread loops of the producer, compiled once per (k-blocks per stage, layout of B):
+    // with those as run-time values the issuing threads measured 8-10 % slower on long-K shapes.
+    auto tma_loop = [&](auto kpb_c, auto bkn_c) -> bool {
+      constexpr int KPB = decltype(kpb_c)::value;
+      constexpr bool BKN = decltype(bkn_c)::value;
+      constexpr int kStage = KPB * C::kKBlockBytes;
       // operand panels are re-read by many CTAs: ask L2 to keep them
       const uint64_t op_pol = (P.l2_hints & 2) ? l2_policy_evict_last() : l2_policy_evict_normal();
+      const bool k3d = KPB > 1 && P.k3d;
       int stage = 0;
       uint32_t phase = 0;
-      bool ok = true;
-      for (int i = 0; ok && i < n_my; ++i) {
+      for (int i = 0; i < n_my; ++i) {
         int d, l, half;
         block_of(i, &d, &l, &half);
         const int mb = d * P.rowsT + l / P.nBn, nb = l % P.nBn;
@@ -1663,85 +1669,79 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
         const int b_row = nb * BN + (half < 0 ? 0 : half * (BN / 2)) + (PAIR ? (int)cta_rank * b_rows : 0);
         const int b_bytes = b_rows * kBK * 2;  // one k-block of them
         const CUtensorMap* const mb2 = half < 0 ? &maps.b : &maps.bh;
-        const CUtensorMap* const mb3 = half < 0 ? &maps.b3 : &maps.bh3;
-        for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
+        const CUtensorMap* const mb3 = BKN ? (half < 0 ? &maps.bkn : &maps.bknh) : (half < 0 ? &maps.b3 : &maps.bh3);
+        for (int kb0 = 0; kb0 < KB; kb0 += KPB) {
           {
             PROF_T0();
             const bool got = mbar_wait(empty_bar(stage), phase ^ 1, P, &sh);
             PROF_ADD(0);
-            if (!got) { ok = false; break; }
+            if (!got) return false;
           }
-          const uint32_t a_dst = smem_base + stage * stage_bytes;
-          const uint32_t b_dst = a_dst + P.kpb * C::kABytes;
+          const uint32_t a_dst = smem_base + stage * kStage;
+          const uint32_t b_dst = a_dst + KPB * C::kABytes;
           // k-blocks of this stage that exist (a ragged last stage is filled, and multiplied, in part)
-          const int nkb = min(P.kpb, KB - kb0);
-          const uint32_t lead_bar = PAIR ? map_to_cta(full_bar(stage), 0) : full_bar(stage);
-          if (P.b_kn) {
-            // B as [K, N]: one box [groups of 64 columns][kpb * 64 k-rows][64], rows past K read as zero;
-            // A as below, k-block by k-block unless its 3-D view exists
-            const uint32_t a_tx = (P.k3d ? P.kpb : nkb) * C::kABytes, b_tx = P.kpb * b_bytes;
-            if (PAIR) {
-              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * (a_tx + b_tx));
-              if (P.k3d) tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
-              else
-                for (int kk = 0; kk < nkb; ++kk)
-                  tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, lead_bar, op_pol);
-              tma_load_3d_pair_hint(b_dst, half < 0 ? &maps.bkn : &maps.bknh, 0, kb0 * kBK, b_row / 64, lead_bar, op_pol);
-            } else {
-              mbar_arrive_expect_tx(full_bar(stage), a_tx + b_tx);
-              if (P.k3d) tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, full_bar(stage), op_pol);
-              else
-                for (int kk = 0; kk < nkb; ++kk)
-                  tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, full_bar(stage), op_pol);
-              tma_load_3d_hint(b_dst, half < 0 ? &maps.bkn : &maps.bknh, 0, kb0 * kBK, b_row / 64, full_bar(stage), op_pol);
-            }
-          } else if (P.k3d) {
-            // one box per operand: [kpb k-blocks][rows][64]; k-blocks past the end of K read as zero
-            if (PAIR) {
-              // both CTAs' bytes are counted on the leader's barrier, which the leader arms
-              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * P.kpb * (C::kABytes + b_bytes));
-              tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
-              tma_load_3d_pair_hint(b_dst, mb3, 0, b_row, kb0, lead_bar, op_pol);
-            } else {
-              mbar_arrive_expect_tx(full_bar(stage), stage_bytes);
-              tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, full_bar(stage), op_pol);
-              tma_load_3d_hint(b_dst, mb3, 0, b_row, kb0, full_bar(stage), op_pol);
-            }
+          const int nkb = KPB == 1 ? 1 : min(KPB, KB - kb0);
+          const uint32_t fbar = full_bar(stage);
+          const uint32_t lead_bar = PAIR ? map_to_cta(fbar, 0) : fbar;
+          // bytes this CTA brings: A as one 3-D box of KPB k-blocks (k-blocks past the end of K read
+          // as zero and count) or k-block by k-block; B [K, N] always as one box of KPB * 64 k-rows
+          const uint32_t a_tx = (k3d ? KPB : nkb) * C::kABytes;
+          const uint32_t b_tx = ((BKN || k3d) ? KPB : nkb) * b_bytes;
+          if (PAIR) {
+            // both CTAs' bytes are counted on the leader's barrier, which the leader arms
+            if (leader) mbar_arrive_expect_tx(fbar, 2 * (a_tx + b_tx));
           } else {
-            if (PAIR) {
-              if (leader) mbar_arrive_expect_tx(full_bar(stage), 2 * nkb * (C::kABytes + b_bytes));
-            } else {
-              mbar_arrive_expect_tx(full_bar(stage), nkb * C::kKBlockBytes);
+            mbar_arrive_expect_tx(fbar, a_tx + b_tx);
+          }
+          if (k3d) {
+            if (PAIR) tma_load_3d_pair_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, lead_bar, op_pol);
+            else tma_load_3d_hint(a_dst, &maps.a3, 0, mb * kBM, kb0, fbar, op_pol);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < KPB; ++kk) {
+              if (kk < nkb) {
+                if (PAIR) tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, lead_bar, op_pol);
+                else tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, (kb0 + kk) * kBK, mb * kBM, fbar, op_pol);
+              }
             }
-            for (int kk = 0; kk < nkb; ++kk) {
-              const int kx = (kb0 + kk) * kBK;
-              if (PAIR) {
-                tma_load_2d_pair_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, lead_bar, op_pol);
-                tma_load_2d_pair_hint(b_dst + kk * b_bytes, mb2, kx, b_row, lead_bar, op_pol);
-              } else {
-                tma_load_2d_hint(a_dst + kk * C::kABytes, &maps.a, kx, mb * kBM, full_bar(stage), op_pol);
-                tma_load_2d_hint(b_dst + kk * C::kBBytes, &maps.b, kx, b_row, full_bar(stage), op_pol);
+          }
+          if (BKN) {
+            // B as [K, N]: one box [groups of 64 columns][KPB * 64 k-rows][64], rows past K read as zero
+            if (PAIR) tma_load_3d_pair_hint(b_dst, mb3, 0, kb0 * kBK, b_row / 64, lead_bar, op_pol);
+            else tma_load_3d_hint(b_dst, mb3, 0, kb0 * kBK, b_row / 64, fbar, op_pol);
+          } else if (k3d) {
+            // one box per operand: [KPB k-blocks][rows][64]
+            if (PAIR) tma_load_3d_pair_hint(b_dst, mb3, 0, b_row, kb0, lead_bar, op_pol);
+            else tma_load_3d_hint(b_dst, mb3, 0, b_row, kb0, fbar, op_pol);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < KPB; ++kk) {
+              if (kk < nkb) {
+                if (PAIR) tma_load_2d_pair_hint(b_dst + kk * b_bytes, mb2, (kb0 + kk) * kBK, b_row, lead_bar, op_pol);
+                else tma_load_2d_hint(b_dst + kk * b_bytes, mb2, (kb0 + kk) * kBK, b_row, fbar, op_pol);
               }
             }
           }
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
       }
-      if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -1); }
-    } else if (warp == kMmaWarp && lane == 0 && leader) {
-      // ---- MMA issuer (the leader CTA issues for the pair) ----
+      return true;
+    };
+    auto mma_loop = [&](auto kpb_c, auto bkn_c) -> bool {
+      constexpr int KPB = decltype(kpb_c)::value;
+      constexpr bool BKN = decltype(bkn_c)::value;
+      constexpr int kStage = KPB * C::kKBlockBytes;
+      constexpr uint32_t kBMajor = BKN ? (1u << 16) : 0u;  // B operand MN-major
+      const uint32_t idesc_full = instr_desc<BN, PAIR ? 256 : 128>() | kBMajor;
+      const uint32_t idesc_half = instr_desc<BN / 2, PAIR ? 256 : 128>() | kBMajor;
+      // K advances by 16 elements per instruction: 32 bytes inside a row (K-major, 2 address units),
+      // 16 rows of 128 bytes (MN-major B)
+      constexpr uint32_t kBStep = BKN ? (kUmmaK * 128) >> 4 : 2;
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
-      const uint32_t b_major_bit = P.b_kn ? (1u << 16) : 0u;
-      const uint32_t idesc_full = instr_desc<BN, PAIR ? 256 : 128>() | b_major_bit;
-      const uint32_t idesc_half = instr_desc<BN / 2, PAIR ? 256 : 128>() | b_major_bit;
-      bool ok = true;
-#ifdef ENTWINE_PROFILE
-      const long long prof_mma0 = clock64();
-#endif
-      for (int i = 0; ok && i < n_my; ++i) {
+      for (int i = 0; i < n_my; ++i) {
         int d_, l_, half;
         block_of(i, &d_, &l_, &half);
         const uint32_t idesc = half < 0 ? idesc_full : idesc_half;
@@ -1750,34 +1750,34 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           PROF_T0();
           const bool got = mbar_wait(tempty_bar(acc), acc_phase ^ 1, P, &sh);
           PROF_ADD(1);
-          if (!got) { ok = false; break; }
+          if (!got) return false;
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb0 = 0; kb0 < KB; kb0 += P.kpb) {
+        for (int kb0 = 0; kb0 < KB; kb0 += KPB) {
           {
             PROF_T0();
             const bool got = mbar_wait(full_bar(stage), phase, P, &sh);
             PROF_ADD(2);
-            if (!got) { ok = false; break; }
+            if (!got) return false;
           }
           tc_fence_after();
-          const uint32_t a_s = smem_base + stage * stage_bytes;
-          const uint32_t b_s = a_s + P.kpb * C::kABytes;
-          const int nkb = min(P.kpb, KB - kb0);
-          for (int kk = 0; kk < nkb; ++kk) {
-            const uint64_t a_desc = smem_desc_sw128(a_s + kk * C::kABytes);
-            // B K-major: k-block kk of this CTA's rows, K advances by 32 bytes inside a row;
-            // B MN-major: k-rows [64 kk, 64 kk + 64) of every 64-column group (groups kpb * 8 KiB
-            // apart), K advances by 16 rows of 128 bytes
-            const uint64_t b_desc = P.b_kn ? smem_desc_sw128_mn(b_s + kk * (kBK * 128), P.kpb * (kBK * 128))
-                                           : smem_desc_sw128(b_s + kk * b_bytes);
-            const uint32_t b_step = P.b_kn ? (kUmmaK * 128) >> 4 : 2;
+          const uint32_t a_s = smem_base + stage * kStage;
+          const uint32_t b_s = a_s + KPB * C::kABytes;
+          const int nkb = KPB == 1 ? 1 : min(KPB, KB - kb0);
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // advancing K by 16 elements = 32 bytes = 2 descriptor address units (K-major)
-              if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + b_step * k, idesc, (kb0 | kk | k) != 0);
-              else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + b_step * k, idesc, (kb0 | kk | k) != 0);
+          for (int kk = 0; kk < KPB; ++kk) {
+            if (kk < nkb) {
+              const uint64_t a_desc = smem_desc_sw128(a_s + kk * C::kABytes);
+              // B K-major: k-block kk of this CTA's rows; B MN-major: k-rows [64 kk, 64 kk + 64) of
+              // every 64-column group (groups KPB * 8 KiB apart)
+              const uint64_t b_desc = BKN ? smem_desc_sw128_mn(b_s + kk * (kBK * 128), KPB * (kBK * 128))
+                                          : smem_desc_sw128(b_s + kk * b_bytes);
+#pragma unroll
+              for (int k = 0; k < kBK / kUmmaK; ++k) {
+                if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + kBStep * k, idesc, (kb0 | kk | k) != 0);
+                else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + kBStep * k, idesc, (kb0 | kk | k) != 0);
+              }
             }
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
@@ -1785,11 +1785,29 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
           else tc_commit(empty_bar(stage));
           if (++stage == n_stages) { stage = 0; phase ^= 1; }
         }
-        if (!ok) break;
         if (PAIR) tc_commit_pair(tfull_bar(acc));  // accumulator complete (both CTAs' halves)
         else tc_commit(tfull_bar(acc));
         if ((acc ^= 1) == 0) acc_phase ^= 1;
       }
+      return true;
+    };
+    using Kpb1 = std::integral_constant<int, 1>;
+    using Kpb2 = std::integral_constant<int, 2>;
+
+    if (warp == kTmaWarp && lane == 0) {
+      // ---- TMA producer (every CTA loads its own operands) ----
+      bool ok;
+      if (P.kpb == 2) ok = P.b_kn ? tma_loop(Kpb2{}, std::true_type{}) : tma_loop(Kpb2{}, std::false_type{});
+      else ok = P.b_kn ? tma_loop(Kpb1{}, std::true_type{}) : tma_loop(Kpb1{}, std::false_type{});
+      if (!ok) { sh.abort = 1; report(P, -ENTWINE_ERR_TIMEOUT, -1); }
+    } else if (warp == kMmaWarp && lane == 0 && leader) {
+      // ---- MMA issuer (the leader CTA issues for the pair) ----
+#ifdef ENTWINE_PROFILE
+      const long long prof_mma0 = clock64();
+#endif
+      bool ok;
+      if (P.kpb == 2) ok = P.b_kn ? mma_loop(Kpb2{}, std::true_type{}) : mma_loop(Kpb2{}, std::false_type{});
+      else ok = P.b_kn ? mma_loop(Kpb1{}, std::true_type{}) : mma_loop(Kpb1{}, std::false_type{});
 #ifdef ENTWINE_PROFILE
       prof_acc_[8] += (unsigned long long)(clock64() - prof_mma0);
 #endif
@@ -2044,7 +2062,7 @@ entwine_fused_kernel(const __grid_constant__ KMaps maps, const KParams P) {
       }
     }
     if (count > 0 && !sh.abort) {
-      consumer_pipeline<NORM, PULL>(P, maps, &sh, smem_base, first, count, on_a, &cnt);
+      consumer_pipeline<NORM, PULL, REG>(P, maps, &sh, smem_base, first, count, on_a, &cnt);
     }
     if (warp == kCommWarp && lane == 0) {
       if (cnt.reduced) atomicAdd(&st->tiles_reduced, (unsigned long long)cnt.reduced);
@@ -2411,10 +2429,13 @@ static cudaError_t order_after_last_launch(DeviceState* d, cudaStream_t stream) 
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-template <int BN, bool PAIR, bool NORM = false, bool PULL = false>
+// The register path of the consumer (KParams::reg_a) is a kernel of its own: with its code compiled
+// into the same kernel, the TMA-ring consumer measured 4-10 us slower on the benchmark's shapes.
+template <int BN, bool PAIR, bool NORM = false, bool PULL = false, bool REG = false>
 static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cudaStream_t stream,
                      bool config_only = false) {
-  if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false>(p, kp, maps, grid, stream, config_only);
+  if (!NORM && !PULL && kp.norm) return launch_bn<BN, PAIR, true, false, REG>(p, kp, maps, grid, stream, config_only);
+  if (!REG && kp.reg_a) return launch_bn<BN, PAIR, NORM, PULL, true>(p, kp, maps, grid, stream, config_only);
   // per device: the shared-memory opt-in has been set, and how many clusters fit at once (shared by
   // all plans, which may be used from different threads)
   static int max_clusters[64] = {0};
@@ -2423,7 +2444,7 @@ static int launch_bn(Plan* p, const KParams& kp, const KMaps& maps, int grid, cu
   int dev = 0;
   CK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ENTWINE_ERR_RESOURCES;
-  auto kern = entwine_fused_kernel<BN, PAIR, NORM, PULL>;
+  auto kern = entwine_fused_kernel<BN, PAIR, NORM, PULL, REG>;
   cudaLaunchConfig_t cfg;
   std::memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(unsigned(grid), 1, 1);
@@ -2484,11 +2505,13 @@ static int ring_geometry(const Plan* p, KParams* kp, bool reg_a) {
   const int kblock_bytes = kBM * kBK * 2 + (p->pair ? 128 : g.BN) * kBK * 2;
   int kpb = p->kpb;
   if (kpb <= 0) {
-    kpb = (kblock_bytes <= 32768 && g.K >= 2 * kBK) ? 2 : 1;
+    // (only with the register consumer, which leaves all of shared memory to the operand ring: beside a
+    // consumer ring, five single k-blocks in flight measured better than two pairs)
+    kpb = (reg_a && kblock_bytes <= 32768 && g.K >= 2 * kBK) ? 2 : 1;
     // a requested number of stages that only fits with single k-blocks gets single k-blocks
     if (kpb == 2 && p->stages > 0 && p->stages * 2 * kblock_bytes + kStagingBytes > kDataBytes) kpb = 1;
   }
-  if (kpb * kblock_bytes > 65536) return ENTWINE_ERR_INVALID;
+  if (kpb > 2 || kpb * kblock_bytes > 65536) return ENTWINE_ERR_INVALID;  // the kernel has loops for 1 and 2
   const int stage_bytes = kpb * kblock_bytes;
   int stages = p->stages;
   if (stages <= 0) {
@@ -2649,7 +2672,7 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  rc = ring_geometry(p, &kp, p->reg_consumer != 0);
+  rc = ring_geometry(p, &kp, p->reg_consumer != 0 || p->consumer_tma == 0);
   if (rc != ENTWINE_OK) return rc;
   kp.prefetch = p->prefetch;
   kp.l2_hints = p->l2_hints;
@@ -2804,7 +2827,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
   kp.list_head_next = d->list_head + size_t((seq_next & 1) ^ 1) * (p->x + 1);
   kp.status_next = &d->status[(seq_next & 1) ^ 1];
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
-  rc = ring_geometry(p, &kp, p->reg_consumer != 0);
+  rc = ring_geometry(p, &kp, p->reg_consumer != 0 || p->consumer_tma == 0);
   if (rc != ENTWINE_OK) return rc;
   kp.prefetch = 0;
   kp.l2_hints = p->l2_hints;
@@ -2991,7 +3014,9 @@ int entwine_plan_set_workspace(entwine_plan_t plan, void* workspace, size_t byte
     KMaps maps;
     std::memset(&maps, 0, sizeof(maps));
     const int grid = std::min(p->num_sms, p->n_gemm_ctas + p->n_comm_ctas);
-    for (int variant = 0; rc == ENTWINE_OK && variant < 3; ++variant) {
+    for (int v6 = 0; rc == ENTWINE_OK && v6 < 6; ++v6) {
+      const int variant = v6 % 3;
+      kp.reg_a = v6 / 3;  // both consumer kernels: options may still change which one a call launches
       kp.norm = variant == 1;
       if (variant == 2) {
         if (p->pair) rc = launch_bn<256, true, false, true>(p, kp, maps, grid, nullptr, true);
@@ -3245,7 +3270,7 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.seq = 0;
   kp.wait_budget_ns = (unsigned long long)p->wait_budget_ns;
   {
-    const int grc = ring_geometry(p, &kp, p->reg_consumer != 0);
+    const int grc = ring_geometry(p, &kp, p->reg_consumer != 0 || p->consumer_tma == 0);
     if (grc != ENTWINE_OK) return grc;
   }
   kp.cws = reinterpret_cast<const __nv_bfloat16*>(base);

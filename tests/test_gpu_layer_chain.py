@@ -89,10 +89,12 @@ def test_layer_chain_matches_oracle(shape):
         oracle_S[(wl.name, r)] = O.out_magnitude_sum(S, Pb, r, W) + np.abs(_vals(res))
         oracle = O.layer_chain_ref(ref_out, I.bits(res), I.bits(w), EPS)
         base = None
-        for order, n_comm, BN in itertools.product((1, 0, 2), (0, 4, 20), (256, 128)):
+        # (reg: the co-located consumer on the shared-memory ring or on the register path)
+        for order, n_comm, BN, reg in itertools.product((1, 0, 2), (0, 4, 20), (256, 128), (0, 1)):
             if N % BN:
                 continue
-            out = _run_and_check(wl, r, order, n_comm, Ad, Bd, Pd, resd, wd, oracle=oracle, block_n=BN)
+            out = _run_and_check(wl, r, order, n_comm, Ad, Bd, Pd, resd, wd, oracle=oracle, block_n=BN,
+                                 reg_consumer=reg)
             if base is None:
                 base = out
             # scheduling never changes a bit of any result

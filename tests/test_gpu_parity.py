@@ -330,9 +330,10 @@ OPTION_SETS = [
     dict(release_group=3), dict(release_group=16), dict(release_group=-1), dict(release_group=-2),
     dict(release_group=5, pair_ctas=0), dict(release_group=-1, colocate=0, tail_help=0),
     # how a stage of the operand ring is filled, and how the co-located consumer moves its tiles
-    dict(kblocks_per_stage=1), dict(kblocks_per_stage=2, stages=2), dict(kblocks_per_stage=1, stages=6),
-    dict(reg_consumer=0), dict(reg_consumer=0, kblocks_per_stage=2, stages=2), dict(reg_consumer=0, kblocks_per_stage=1),
-    dict(reg_consumer=0, pair_ctas=0), dict(reg_consumer=1, pair_ctas=0, kblocks_per_stage=1),
+    dict(kblocks_per_stage=1), dict(kblocks_per_stage=2, stages=2), dict(kblocks_per_stage=1, stages=6, reg_consumer=1),
+    dict(reg_consumer=1), dict(reg_consumer=1, kblocks_per_stage=2, stages=2), dict(reg_consumer=1, kblocks_per_stage=1),
+    dict(reg_consumer=1, stages=2), dict(reg_consumer=1, l2_hints=0), dict(reg_consumer=1, release_group=-1),
+    dict(reg_consumer=0, pair_ctas=0), dict(reg_consumer=1, pair_ctas=0), dict(reg_consumer=1, pair_ctas=0, kblocks_per_stage=1),
     dict(split_last_wave=0), dict(consumer_tma=0), dict(consumer_tma=0, tail_help=0, colocate=0),
 ]
 
@@ -439,7 +440,7 @@ def test_leading_dimensions(wl):
     Bpad[:, :wl.K] = Bd
     r = 1
     res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, 256, 1, 4)
-    for opts in (dict(), dict(kblocks_per_stage=1), dict(pair_ctas=0)):
+    for opts in (dict(), dict(kblocks_per_stage=2), dict(reg_consumer=1), dict(pair_ctas=0)):
         p0 = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, **opts)
         out0, send0 = _alloc_outputs(wl)
         p0.gemm_rs(Ad, Bd, Pd, out0, send0)
@@ -482,7 +483,7 @@ def test_b_given_as_k_by_n(wl):
     r = wl.W - 1
     BN = 256 if wl.N % 256 == 0 else 128
     res = O.gemm_rs(Ab, Bb, Pb, r, wl.W, BN, 1, 4)
-    for opts in (dict(), dict(pair_ctas=0), dict(kblocks_per_stage=1), dict(block_n=128)):
+    for opts in (dict(), dict(pair_ctas=0), dict(kblocks_per_stage=2), dict(reg_consumer=1), dict(block_n=128)):
         p0 = E.Plan(wl.M, wl.N, wl.K, wl.W, E.ORDER_INTERLEAVED, 4, rank=r, **opts)
         out0, send0 = _alloc_outputs(wl)
         p0.gemm_rs(Ad, Bd, Pd, out0, send0)
