@@ -787,7 +787,7 @@ def main():
     roof["traffic_source"] = NCU_TRAFFIC.get(wl.name, {}).get("summary")
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
     roof["roofline_us"] = max(t_tc, t_hbm) * 1e6
-    roof["kernel"] = "entwine_fused_kernel<256, true, false, false>"
+    roof["kernel"] = "entwine_fused_kernel<256, true, false, false, false>"
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
