@@ -34,9 +34,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # the ncu capture of the named workload that profiles/ summarises; the summary file is carried
 # beside the number so that a stale figure can be told from a fresh one.
 NCU_TRAFFIC = {
-    "attn_out_proj": {"bytes": 53.69e6, "summary": "profiles/fused_kernel_attn_out_proj.md"},
-    "mlp_down_proj": {"bytes": 845.38e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
-    "short_k_comm_bound": {"bytes": 507.35e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+    "attn_out_proj": {"bytes": 55.75e6, "summary": "profiles/fused_kernel_attn_out_proj.md"},
+    "mlp_down_proj": {"bytes": 830.84e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+    "short_k_comm_bound": {"bytes": 514.77e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
 }
 # Launch configuration per workload: communication SMs, tile order.
 # Launch configuration per workload (the best point of a budget x order scan on B200): number of
@@ -783,6 +783,12 @@ def main():
     # cap, and the nominal HBM bandwidth
     t_alt = max(wl.flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12), wl.comm_bytes / 8.0e12)
     roof["frac_vs_sustained_tensor_and_nominal_hbm"] = t_alt / (mean_us * 1e-6)
+    if tensor_bound and kernel_mhz:
+        # tensor-pipe cycles the FLOPs need (148 SMs x 8192 dense bf16 FLOP per cycle and SM: one
+        # 128 x 256 x 16 tcgen05.mma per 128 cycles) over the cycles the call took at the clock measured
+        # inside the kernel: the fraction with the power-limited clock taken out
+        props = torch.cuda.get_device_properties(torch.cuda.current_device())
+        roof["tensor_cycles_ideal_over_measured"] = (wl.flops / (props.multi_processor_count * 8192.0)) / (mean_us * kernel_mhz)
     roof["traffic"] = NCU_TRAFFIC.get(wl.name, {}).get("bytes")
     roof["traffic_source"] = NCU_TRAFFIC.get(wl.name, {}).get("summary")
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
