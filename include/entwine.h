@@ -375,7 +375,9 @@ int entwine_last_sm_clock(entwine_plan_t plan, int64_t out[2]);
  * a device-side timeout or index failure of that call then goes unnoticed (its outputs are
  * incomplete), so pass status_out wherever the result matters.  Options that this entry point
  * does not implement (a release group other than 1, a withheld peer flag) make it return
- * ENTWINE_ERR_INVALID.
+ * ENTWINE_ERR_INVALID, and so does a `stream` that is being captured into a CUDA graph (every call
+ * uploads the plan's tables from host memory; for graphs use entwine_plan_set_workspace and
+ * entwine_gemm_rs).
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
  * caches it per device: make that first call outside any stream capture.  All calls on a

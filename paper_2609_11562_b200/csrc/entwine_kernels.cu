@@ -3202,6 +3202,16 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
   // options this entry point does not implement are refused, not ignored
   if (p->release_group != 1 || p->withhold_peer >= 0) return ENTWINE_ERR_INVALID;
+  {
+    // every call uploads the plan's tables from the plan's host vectors: captured into a graph,
+    // those copies would keep host addresses that a later option change frees
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess) {
+      cudaGetLastError();
+      return ENTWINE_ERR_CUDA;
+    }
+    if (cs != cudaStreamCaptureStatusNone) return ENTWINE_ERR_INVALID;
+  }
 
   // ---- sizes against the static maximum ----
   const size_t c_bytes = size_t(g.M) * g.N * 2;

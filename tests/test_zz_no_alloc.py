@@ -127,3 +127,13 @@ def test_static_scratch_rejects_what_it_cannot_do():
         plan.gemm_rs_static(dummy, dummy, dummy, dummy, dummy)
     assert e.value.code == E.ERR_INVALID
     plan.destroy()
+    # a capturing stream is refused (the call uploads tables from host memory), and the capture survives it
+    plan = E.Plan(small.M, small.N, small.K, small.W, E.ORDER_INTERLEAVED, 4)
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s):
+        with pytest.raises(E.EntwineError) as e:
+            plan.gemm_rs_static(dummy, dummy, dummy, dummy, dummy, stream=s, want_status=False)
+        dummy.add_(0)
+    assert e.value.code == E.ERR_INVALID
+    plan.destroy()
