@@ -700,6 +700,8 @@ def main():
         dist.barrier()
     torch.cuda.synchronize()
     wall = time.perf_counter() - t_wall0
+    status = plan.last_status()
+    kernel_mhz = plan.last_sm_clock_mhz()  # cycle counter against the global timer inside the last timed launch
     # A short timed region can end before nvidia-smi's next sample: keep the same load running,
     # untimed, until two samples under load exist.
     extended = False
@@ -714,8 +716,6 @@ def main():
     clocks["sampled"] = ("during the timed region" if not extended else
                          "timed region shorter than the sampling period: same load continued untimed")
     us = [a.elapsed_time(b) * 1e3 for a, b in evs]
-    status = plan.last_status()
-    kernel_mhz = plan.last_sm_clock_mhz()  # cycle counter against the global timer inside the last timed launch
     total_us = max_over_ranks(sum(us), dist, "cuda")
     mean_us = total_us / args.steps
     value = whole_job_tflops(world, wl.flops, mean_us * 1e-6)
@@ -786,9 +786,10 @@ def main():
     if tensor_bound and kernel_mhz:
         # tensor-pipe cycles the FLOPs need (148 SMs x 8192 dense bf16 FLOP per cycle and SM: one
         # 128 x 256 x 16 tcgen05.mma per 128 cycles) over the cycles the call took at the clock measured
-        # inside the kernel: the fraction with the power-limited clock taken out
+        # inside the kernel (the last timed launch: its own time and its own clock): the fraction with the
+        # power-limited clock taken out
         props = torch.cuda.get_device_properties(torch.cuda.current_device())
-        roof["tensor_cycles_ideal_over_measured"] = (wl.flops / (props.multi_processor_count * 8192.0)) / (mean_us * kernel_mhz)
+        roof["tensor_cycles_ideal_over_measured"] = (wl.flops / (props.multi_processor_count * 8192.0)) / (us[-1] * kernel_mhz)
     roof["traffic"] = NCU_TRAFFIC.get(wl.name, {}).get("bytes")
     roof["traffic_source"] = NCU_TRAFFIC.get(wl.name, {}).get("summary")
     roof["peak_source"] = peaks["_source"] + (" burst" if tensor_bound else "")
@@ -807,7 +808,7 @@ def main():
                    "emulated_rank": launch["rank"], "l2": "flushed between timed steps (512 MiB memset)",
                    "multi_gpu": "replicas only"},
         "us_per_call": {"mean": mean_us, "median": statistics.median(us), "min": min(us),
-                        "sm_mhz_inside_kernel": kernel_mhz, "mean_us_times_sm_mhz": mean_us * kernel_mhz},
+                        "last_us": us[-1], "sm_mhz_inside_last_kernel": kernel_mhz, "last_us_times_sm_mhz": us[-1] * kernel_mhz},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roof,
         "device_status": {"t_gemm_us": status["t_gemm_ns"] / 1e3, "t_end_us": status["t_end_ns"] / 1e3,
                           "tail_us": (status["t_end_ns"] - status["t_gemm_ns"]) / 1e3},
@@ -832,7 +833,7 @@ def main():
                 "fused_graph_replay_us": r["fused_graph_replay_us"],
                 "roofline_us": max(tc, hb) * 1e6, "roofline_frac": max(tc, hb) * 1e6 / fused,
                 "roofline_frac_back_to_back": max(tc, hb) * 1e6 / r["fused_back_to_back_us"],
-                "sm_mhz_inside_kernel": r["sm_mhz"], "fused_us_times_sm_mhz": fused * r["sm_mhz"],
+                "sm_mhz_inside_last_kernel": r["sm_mhz"], "last_fused_us_times_sm_mhz": r["fused_us"][-1] * r["sm_mhz"],
                 "bound": "tensor" if tc >= hb else "hbm",
                 "unfused_cublas_then_reduce_us": med(r["unfused_us"]),
                 "speedup_vs_unfused": med(r["unfused_us"]) / fused,
