@@ -84,6 +84,7 @@ struct Plan {
   int kpb = 0;              // k-blocks (64 elements of K) per stage, 0 = choose
   int split_opt = 1;        // a last wave that fills at most half of the CTA pairs runs as half-width units
   int64_t lda = 0, ldb = 0; // leading dimensions of A and B in elements, 0 = contiguous
+  int peers_compact = 0;    // (set around a launch by the host-buffer calls) peers are staged as [W-1][R][N]
   int b_kn = 0;             // 1: B is [K_local, N] (N contiguous) instead of [N, K_local]
   int colocate = 1;         // consumer warps of a producer CTA work while it produces
   int reg_consumer = 0;     // 1: ... from registers (plain loads and stores) instead of a shared-memory TMA ring

@@ -158,7 +158,10 @@ struct KParams {
   __nv_bfloat16* out;            // out_shard [R][N] (written by the reducing warps)
   const __nv_bfloat16* cws;      // the rank's partial C [M][N] as the consumer reads it (register path)
   __nv_bfloat16* cws_out;        // ... as the producer's epilogue writes it
-  const __nv_bfloat16* peers;    // incoming partials [W-1][M][N] (register path; pull mode: see heap)
+  const __nv_bfloat16* peers;    // incoming partials [W-1][peer_rows][N] (register path; pull mode: see heap)
+  int peer_row0;                 // row of the [M,N] numbering that is row 0 of a peer's plane: 0 for the
+  int peer_rows;                 // full [W-1][M][N] layout (peer_rows = M), r * R for the compact staging
+                                 // of the host-buffer calls, which holds partition r's rows only (= R)
   __nv_bfloat16* send;           // send_bufs [W-1][R][N] (register path)
   long long heap_buf_off;        // pull mode: offset of this call's partial-output buffer inside a segment
   unsigned* flags_own;           // [W][Q]
@@ -703,7 +706,8 @@ __device__ __forceinline__ const __nv_bfloat16* peer_base(const KParams& P, int 
     const int w = q + (q >= P.r ? 1 : 0);
     return reinterpret_cast<const __nv_bfloat16*>(P.heap + (long long)w * P.heap_stride + P.heap_buf_off);
   }
-  return P.peers + (long long)q * P.M * P.N;
+  // (rows are numbered as in [M,N]: the offset of the plane's first row is taken out here)
+  return P.peers + ((long long)q * P.peer_rows - P.peer_row0) * P.N;
 }
 // ReduceTile of Sec. 4.2 on a whole tile: local contribution first, then the peers in ascending rank
 // order, fp32, one rounding.  A thread's 8 chunks go in batches of 16 / W chunks: all loads of a
@@ -1215,7 +1219,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             if (nkind == 0) {
               for (int q = lane - 1; q >= 0 && q < P.W - 1; q += 31) {
                 if (P.skip_wait || ld_acquire_gpu(&P.flags_peer[q * P.Q + nt]) >= P.epoch)
-                  tma_prefetch_l2_2d(&maps.p_pf, ncol, q * P.M + nrow);
+                  tma_prefetch_l2_2d(&maps.p_pf, ncol, q * P.peer_rows + nrow - P.peer_row0);
               }
             }
           }
@@ -1308,8 +1312,8 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
                 // as one 3-D box
                 tma_load_2d_hint(dst, &maps.c_ld[ring.geom], col, src_row + step * rows, ring.full(slot), pol);
                 if (!PULL) {
-                  tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col, src_row + step * rows, 0,
-                                   ring.full(slot), pol);
+                  tma_load_3d_hint(dst + ring.sub_bytes, &maps.p_ld[ring.geom], col,
+                                   src_row + step * rows - P.peer_row0, 0, ring.full(slot), pol);
                 } else {
                   // the peers' rows come straight from their segments of the heap: the ranks
                   // below this one, then the ranks above it, each group as one 3-D box
@@ -2724,13 +2728,17 @@ static int launch(Plan* p, int mode, const void* A, const void* B, const void* p
   bool ok = (mode != MODE_COMM_ONLY)
                 ? make_operand_maps(&maps, a_p, b_p, g, pair ? 128 : g.BN, kp.kpb, p->lda, p->ldb, kp.b_kn = p->b_kn, &kp.k3d)
                 : (make_map(&maps.a, a_p, g.M, g.N, kBK, kBM, true) && make_map(&maps.b, b_p, g.M, g.N, kBK, kBM, true));
-  ok = ok && make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * g.M : g.M, g.N, kTile, kTile, false);
+  // rows of one peer's plane: all M, or (compact staging of the host-buffer calls) partition r's R
+  const int64_t prows = p->peers_compact ? g.R : g.M;
+  kp.peer_rows = int(prows);
+  kp.peer_row0 = p->peers_compact ? int(p->rank * g.R) : 0;
+  ok = ok && make_map(&maps.p_pf, comm ? peers : d->C, comm ? int64_t(g.W - 1) * prows : g.M, g.N, kTile, kTile, false);
   for (int id = 0; ok && id < 2; ++id) {
     const int rs = kp.rs[id];
     const int prs = kp.prs[id];
     ok = make_map(&maps.c_ld[id], c_src, g.M, g.N, kTile, rs, false) &&
          make_map(&maps.c_push[id], c_src, g.M, g.N, kTile, prs, false) &&
-         (comm ? make_map3(&maps.p_ld[id], peers, g.W - 1, g.M, g.N, kTile, rs, g.W - 1)
+         (comm ? make_map3(&maps.p_ld[id], peers, g.W - 1, prows, g.N, kTile, rs, g.W - 1)
                : make_map3(&maps.p_ld[id], d->C, 1, g.M, g.N, kTile, rs, 1)) &&
          make_map(&maps.send_st[id], comm ? send : d->C, comm ? int64_t(g.W - 1) * g.R : g.M, g.N, kTile, prs, false) &&
          make_map(&maps.res_ld[id], norm ? norm->residual : d->C, norm ? g.R : g.M, g.N, kTile, prs, false) &&
@@ -3054,7 +3062,8 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, cons
   DeviceState* d = plan->dev;
   const Geometry& g = plan->g;
   const size_t szA = size_t(g.M) * g.K * 2, szB = size_t(g.N) * g.K * 2;
-  const size_t szP = size_t(g.W - 1) * g.M * g.N * 2, szO = size_t(g.R) * g.N * 2;
+  // staging of the incoming partials is compact: [W-1][R][N], the rows of partition r that the call reads
+  const size_t szP = size_t(g.W - 1) * g.R * g.N * 2, szO = size_t(g.R) * g.N * 2;
   const size_t szS = size_t(g.W - 1) * g.R * g.N * 2;
   if (!d->own_stream) {
     CK(cudaStreamCreateWithFlags(&d->own_stream, cudaStreamNonBlocking));
@@ -3073,14 +3082,16 @@ int entwine_gemm_rs_host(entwine_plan_t plan, const void* A, const void* B, cons
   const size_t part = size_t(g.R) * g.N * 2, full = size_t(g.M) * g.N * 2;
   for (int q = 0; q < g.W - 1; ++q) {
     const size_t off = size_t(q) * full + size_t(plan->rank) * part;
-    CK(cudaMemcpyAsync(reinterpret_cast<char*>(d->sPeers) + off, static_cast<const char*>(peer_partials) + off,
+    CK(cudaMemcpyAsync(reinterpret_cast<char*>(d->sPeers) + size_t(q) * part, static_cast<const char*>(peer_partials) + off,
                        part, cudaMemcpyHostToDevice, s));
   }
   {
     // the staging copies are contiguous whatever the leading dimensions of device operands are
     const int64_t lda = plan->lda, ldb = plan->ldb;
     plan->lda = plan->ldb = 0;
+    plan->peers_compact = 1;
     rc = launch(plan, MODE_FUSED, d->sA, d->sB, nullptr, d->sPeers, d->sOut, d->sSend, 0, s);
+    plan->peers_compact = 0;
     plan->lda = lda;
     plan->ldb = ldb;
   }
@@ -3100,7 +3111,8 @@ int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B
   DeviceState* d = plan->dev;
   const Geometry& g = plan->g;
   const size_t szA = size_t(g.M) * g.K * 2, szB = size_t(g.N) * g.K * 2;
-  const size_t szP = size_t(g.W - 1) * g.M * g.N * 2, szO = size_t(g.R) * g.N * 2;
+  // staging of the incoming partials is compact: [W-1][R][N], the rows of partition r that the call reads
+  const size_t szP = size_t(g.W - 1) * g.R * g.N * 2, szO = size_t(g.R) * g.N * 2;
   const size_t szS = size_t(g.W - 1) * g.R * g.N * 2;
   if (!d->pipe) {
     DeviceState::HostPipe* hp = new DeviceState::HostPipe();
@@ -3132,7 +3144,7 @@ int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B
   const size_t part = size_t(g.R) * g.N * 2, full = size_t(g.M) * g.N * 2;
   for (int q = 0; q < g.W - 1; ++q) {
     const size_t off = size_t(q) * full + size_t(plan->rank) * part;
-    CK(cudaMemcpyAsync(reinterpret_cast<char*>(hp->peers[s]) + off, static_cast<const char*>(peer_partials) + off,
+    CK(cudaMemcpyAsync(reinterpret_cast<char*>(hp->peers[s]) + size_t(q) * part, static_cast<const char*>(peer_partials) + off,
                        part, cudaMemcpyHostToDevice, hp->up));
   }
   CK(cudaEventRecord(hp->up_done[s], hp->up));
@@ -3142,7 +3154,9 @@ int entwine_gemm_rs_host_begin(entwine_plan_t plan, const void* A, const void* B
   {
     const int64_t lda = plan->lda, ldb = plan->ldb;
     plan->lda = plan->ldb = 0;
+    plan->peers_compact = 1;
     rc = launch(plan, MODE_FUSED, hp->A[s], hp->B[s], nullptr, hp->peers[s], hp->out[s], hp->send[s], 0, hp->comp);
+    plan->peers_compact = 0;
     plan->lda = lda;
     plan->ldb = ldb;
   }
@@ -3286,6 +3300,8 @@ extern "C" int entwine_gemm_rs_static(entwine_plan_t plan, const void* A, const 
   kp.cws = reinterpret_cast<const __nv_bfloat16*>(base);
   kp.cws_out = reinterpret_cast<__nv_bfloat16*>(base);
   kp.peers = static_cast<const __nv_bfloat16*>(peer_partials);
+  kp.peer_rows = g.M;
+  kp.peer_row0 = 0;
   kp.send = static_cast<__nv_bfloat16*>(send_bufs);
   kp.prefetch = p->prefetch;
   kp.l2_hints = p->l2_hints;
