@@ -2294,8 +2294,21 @@ static WorkspaceLayout workspace_layout(const Plan* p) {
   return w;
 }
 
-static int ensure_device(Plan* p) {
-  if (p->dev) return ENTWINE_OK;
+// The partial-output workspace C[M,N] of a plan that allocates its own memory is allocated when a
+// call first needs it: pull mode keeps its partial in the heap and never does.
+static int ensure_partial_c(Plan* p) {
+  DeviceState* d = p->dev;
+  if (d->C) return ENTWINE_OK;
+  const size_t bytes = size_t(p->g.M) * p->g.N * 2;
+  if (cudaMalloc(&d->C, bytes) != cudaSuccess || cudaMemset(d->C, 0, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return ENTWINE_ERR_CUDA;
+  }
+  return ENTWINE_OK;
+}
+
+static int ensure_device(Plan* p, bool need_c = true) {
+  if (p->dev) return need_c ? ensure_partial_c(p) : ENTWINE_OK;
   int sms = device_sm_count();
   if (sms <= 0) return ENTWINE_ERR_CUDA;
   int dev = 0;
@@ -2332,7 +2345,7 @@ static int ensure_device(Plan* p) {
          cudaMemcpy(d->list_offs_pull, t.pull_list_offs.data(), t.pull_list_offs.size() * 4, cudaMemcpyHostToDevice) ==
              cudaSuccess;
   } else {
-    ok = cudaMalloc(&d->C, size_t(g.M) * g.N * 2) == cudaSuccess &&
+    ok = (!need_c || cudaMalloc(&d->C, size_t(g.M) * g.N * 2) == cudaSuccess) &&
          cudaMalloc(&d->flags_own, n_own * 4) == cudaSuccess &&
          cudaMalloc(&d->flags_peer, n_peer * 4) == cudaSuccess &&
          cudaMalloc(&d->tasks, t.dev_tasks.size() * sizeof(Task)) == cudaSuccess &&
@@ -2347,7 +2360,7 @@ static int ensure_device(Plan* p) {
     init[0].t_start = init[1].t_start = ~0ULL;
     ok = cudaMemset(d->flags_own, 0, n_own * 4) == cudaSuccess &&
          cudaMemset(d->flags_peer, 0xff, n_peer * 4) == cudaSuccess &&
-         cudaMemset(d->C, 0, size_t(g.M) * g.N * 2) == cudaSuccess &&
+         (!d->C || cudaMemset(d->C, 0, size_t(g.M) * g.N * 2) == cudaSuccess) &&
          cudaMemcpy(d->tasks, t.dev_tasks.data(), t.dev_tasks.size() * sizeof(Task),
                     cudaMemcpyHostToDevice) == cudaSuccess &&
          cudaMemcpy(d->list_offs, t.list_offs.data(), t.list_offs.size() * 4, cudaMemcpyHostToDevice) ==
@@ -2561,7 +2574,7 @@ struct NormArgs {
 
 static int launch(Plan* p, int mode, const void* A, const void* B, const void* partial, const void* peers,
                   void* out, void* send, int n_ctas, cudaStream_t stream, const NormArgs* norm = nullptr) {
-  if (!p->dev || !(p->launched || p->dev->user_ws)) {
+  if (!p->dev || !p->dev->C || !(p->launched || p->dev->user_ws)) {
     // the first launch allocates the workspace and configures the kernel: not inside a capture
     // (a plan with a caller-provided workspace did both in entwine_plan_set_workspace)
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -2779,7 +2792,7 @@ static int launch_pull(Plan* p, const void* A, const void* B, void* heap, int64_
     return ENTWINE_ERR_CUDA;
   }
   if (cap != cudaStreamCaptureStatusNone) return ENTWINE_ERR_INVALID;  // the epoch is a launch parameter
-  int rc = ensure_device(p);
+  int rc = ensure_device(p, /*need_c=*/false);  // the partial output lives in the heap
   if (rc != ENTWINE_OK) return rc;
   DeviceState* d = p->dev;
   const Geometry& g = p->g;
