@@ -118,8 +118,9 @@ enum {
                                       memory they leave goes to the co-located consumer ring;
                                       0 (default): chosen from the shape                         */
   ENTWINE_OPT_KBLOCKS_PER_STAGE = 15, /* k-blocks (64 elements of K_local) per stage of the operand
-                                      ring: 1 or 2; 0 (default): 2 where a k-block of both operands
-                                      is 32 KiB (CTA pairs, BN = 128), else 1.  With 2 and K_local a
+                                      ring: 1 or 2; 0 (default): 1 beside the consumer's TMA ring; 2
+                                      with the register consumer where a k-block of both operands
+                                      is 32 KiB (CTA pairs, BN = 128).  With 2 and K_local a
                                       multiple of 64 an operand's share of a stage arrives as one
                                       32 KiB TMA box                                                */
   ENTWINE_OPT_LDA             = 16, /* leading dimension of A in elements (row pitch), a multiple of 8
