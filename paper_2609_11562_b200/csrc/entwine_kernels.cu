@@ -1445,13 +1445,21 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
     const uint64_t pol = (P.l2_hints & 1) ? l2_policy_evict_first() : l2_policy_evict_normal();
     unsigned long long pend = 0;  // queue of barrier addresses' slot/ring ids, 8 bits each
     int n_pend = 0;
+    // returns the oldest pushed slot: its store has read it (awaited by the caller) and the reducing
+    // warps have passed it (they only read a pushed slot's record, so the store does not wait for
+    // them: the slot's return does)
+    auto retire_one = [&]() {
+      const Ring rr = make_ring<REG>(smem_base, int(pend >> 4) & 1, P, sh);
+      const int sl = int(pend & 15u);
+      if (!mbar_wait(rr.red(sl), uint32_t(pend >> 5) & 1u, P, sh)) sh->abort = 1;
+      mbar_arrive(rr.empty(sl));
+      pend >>= 8;
+      --n_pend;
+    };
     auto retire_all = [&]() {
       if (!n_pend) return;
       bulk_wait_read<0>();
-      for (; n_pend > 0; --n_pend, pend >>= 8) {
-        const Ring rr = make_ring<REG>(smem_base, int(pend >> 4) & 1, P, sh);
-        mbar_arrive(rr.empty(int(pend & 15u)));
-      }
+      while (n_pend > 0) retire_one();
     };
     int slot = -1;
     uint32_t ph = 0;
@@ -1474,11 +1482,11 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         continue;
       }
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
-      if (!mbar_wait(ring.red(slot), ph, P, sh)) {
-        sh->abort = 1;
-        break;
-      }
       if (m.kind == 0 || (REG && m.kind >= 4) || (NORM && (m.kind == 2 || m.kind == 3))) {
+        if (!mbar_wait(ring.red(slot), ph, P, sh)) {
+          sh->abort = 1;
+          break;
+        }
         if (NORM && ((m.kind == 0 && m.aux >= 0) || (REG && m.kind == 4))) {
           // layer chain: the last step of a reduce task (or a whole task done from registers,
           // whose first destination row is dst_y) counts its tile in the band
@@ -1491,12 +1499,10 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         bulk_commit();
         if (n_pend == kPend) {
           bulk_wait_read<kPend - 1>();  // the oldest store has read its slot
-          const Ring rr = make_ring<REG>(smem_base, int(pend >> 4) & 1, P, sh);
-          mbar_arrive(rr.empty(int(pend & 15u)));
-          pend >>= 8;
-          --n_pend;
+          retire_one();
+          if (sh->abort) break;
         }
-        pend |= (unsigned long long)(unsigned(slot) | (unsigned(ring.id) << 4)) << (8 * n_pend);
+        pend |= (unsigned long long)(unsigned(slot) | (unsigned(ring.id) << 4) | (ph << 5)) << (8 * n_pend);
         ++n_pend;
       }
     }
