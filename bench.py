@@ -34,9 +34,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # the ncu capture of the named workload that profiles/ summarises; the summary file is carried
 # beside the number so that a stale figure can be told from a fresh one.
 NCU_TRAFFIC = {
-    "attn_out_proj": {"bytes": 55.75e6, "summary": "profiles/fused_kernel_attn_out_proj.md"},
-    "mlp_down_proj": {"bytes": 830.84e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
-    "short_k_comm_bound": {"bytes": 514.77e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+    "attn_out_proj": {"bytes": 55.89e6, "summary": "profiles/fused_kernel_attn_out_proj.md"},
+    "mlp_down_proj": {"bytes": 826.88e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
+    "short_k_comm_bound": {"bytes": 514.21e6, "summary": "profiles/fused_kernel_mlp_down_and_short_k.md"},
 }
 # Launch configuration per workload: communication SMs, tile order.
 # Launch configuration per workload (the best point of a budget x order scan on B200): number of
