@@ -85,6 +85,12 @@ constexpr int kStagingBytes = 4 * kEpiWarpBytes;
 constexpr int kRingBOff = 0;
 constexpr int kRingBBytes = 196608;
 constexpr int kMaxSlots = 8;
+#ifndef ENTWINE_NORM_LOADS
+#define ENTWINE_NORM_LOADS 1
+#endif
+// Layer chain: 1: the reducing warps read the tile to normalise themselves (from L2, eight 16-byte loads per
+// thread in flight; the ring slot carries the task only); 0: its rows come into the slot by TMA.
+constexpr bool kNormLoads = ENTWINE_NORM_LOADS != 0;
 constexpr int kRegSlots = 4;       // task descriptors in flight between the claiming and the reducing warps
 constexpr int kMaxStages = 6;
 constexpr int kBarOff = kDataBytes;
@@ -941,7 +947,7 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
         const int g = ctid + k * kRedThreads;
         if (g >= g0 && g < g1) resv[k] = ld_shared_v4(sbase + (g - g0) * 16);
       }
-    } else if (NORM && m.kind == 2) {
+    } else if (NORM && (m.kind == 2 || m.kind == 6)) {
       // Normalisation of prs rows of one 128 x 128 tile of a complete band; the rows are in the
       // slot (loaded from hidden_out by TMA).  m.aux >= 0: the first step of a run of tiles of
       // band m.aux: 1/RMS of the band's 128 rows from the nTn partial sums of each row, kept in
@@ -976,7 +982,29 @@ __device__ __forceinline__ void reducer_role(const KParams& P, CtaShared* sh, ui
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
       float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       acc_bf16x8(w, __ldg(reinterpret_cast<const uint4*>(P.weight + m.dst_x + (ctid & 15) * 8)));
-      const int n_chunks = ring.prs * (kTile * 2 / 16);
+      if (m.kind == 6) {
+        // the whole 128 x 128 tile from L2 (hidden_out was stored there by the reduce tasks; the claiming
+        // warp acquired the band's count before it handed this record over): this thread's eight
+        // chunks, rows ctid / 16 + 16 k, all loads in flight before the first is used
+        const __nv_bfloat16* src = P.out + (long long)m.dst_y * P.N + m.dst_x + (ctid & 15) * 8;
+        __nv_bfloat16* dst = P.norm_out + (long long)m.dst_y * P.N + m.dst_x + (ctid & 15) * 8;
+        // (the registers that hold a tile's residual during its reduce steps are free here: every reduce
+        // task reloads them before it uses them)
+        uint4 (&v)[kResChunks] = resv;
+#pragma unroll
+        for (int k = 0; k < kResChunks; ++k) v[k] = ld_l2_v4(src + (long long)((ctid >> 4) + k * (kRedThreads / 16)) * P.N);
+#pragma unroll
+        for (int k = 0; k < kResChunks; ++k) {
+          const int row = (ctid >> 4) + k * (kRedThreads / 16);
+          float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          acc_bf16x8(h, v[k]);
+          const float inv = sh->inv_rms[row];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) h[e] = h[e] * inv * w[e];
+          __stcs(reinterpret_cast<uint4*>(dst + (long long)row * P.N), pack_bf16x8(h));
+        }
+      }
+      const int n_chunks = m.kind == 6 ? 0 : ring.prs * (kTile * 2 / 16);
       for (int c = ctid; c < n_chunks; c += kRedThreads) {
         const int row = m.dst_y + (c >> 4);  // row of hidden_out; its band row is row % 128
         float h[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -1065,6 +1093,21 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
             run_ok = wait_count(&P.band_ctr[band], (unsigned)P.nTn, P);
             if (!run_ok) break;
             fence_async_all();  // the TMA reads of hidden_out are ordered after the acquire
+          }
+          if (kNormLoads) {
+            // one record per tile: the reducing warps fetch its rows themselves
+            const int slot = it % ring.n_slots;
+            run_ok = mbar_wait(ring.empty(slot), ((it / ring.n_slots) & 1) ^ 1, P, sh);
+            if (!run_ok) break;
+            SlotMeta& m = sh->meta[ring.id][slot];
+            m.kind = 6;
+            m.dst_x = tc * kTile;
+            m.dst_y = band * kTile;
+            m.aux = (band != band_seen) ? band : -1;
+            band_seen = band;
+            mbar_arrive(ring.full(slot));
+            it += 1;
+            continue;
           }
           for (int u = 0; run_ok && u < kTile / ring.prs; ++u) {
             const int slot = it % ring.n_slots;
@@ -1482,7 +1525,7 @@ __device__ __forceinline__ void consumer_pipeline(const KParams& P, const KMaps&
         continue;
       }
       const uint32_t sbase = ring.base + slot * ring.slot_bytes;
-      if (m.kind == 0 || (REG && m.kind >= 4) || (NORM && (m.kind == 2 || m.kind == 3))) {
+      if (m.kind == 0 || (REG && m.kind >= 4) || (NORM && (m.kind == 2 || m.kind == 3 || m.kind == 6))) {
         if (!mbar_wait(ring.red(slot), ph, P, sh)) {
           sh->abort = 1;
           break;
